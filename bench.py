@@ -1,0 +1,318 @@
+#!/usr/bin/env python
+"""Benchmark of the CLEAR attention forward pass (one call = one attention layer of one denoising step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is effective TFLOP/s, 4 * sum(M) * head_dim * H * B / time (the paper's
+4 * sum(M) * c), with q, k, v resident in HBM; `e2e` is the same metric through the host-tensor C-ABI
+entry point with the host<->device copies inside the timed region.  With N > 1 (torchrun) every rank runs
+an independent replica of the workload on its own GPU: the path has no exchange step.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2412_16112_b200 import workloads
+
+METRIC = "effective TFLOP/s (4*sum(M)*c) of the CLEAR attention forward"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons for one GPU while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                parts = [x.strip() for x in out.strip().split(",")]
+                if len(parts) >= 7:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        self._thread.join(timeout=10)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            try:
+                sm.append(float(s[0]))
+                mx.append(float(s[1]))
+            except ValueError:
+                continue
+            for n, val in zip(names, s[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def sample_rows_for_cpu(w, n_text_rows, n_img_rows, seed=0):
+    rng = np.random.default_rng(seed)
+    n = w.grid_h * w.grid_w
+    rows = [(0, 0, int(i)) for i in rng.integers(0, max(w.n_text, 1), n_text_rows) if w.n_text > 0]
+    rows += [(0, 0, w.n_text + int(p)) for p in rng.integers(0, n, n_img_rows)]
+    return np.array(rows, dtype=np.int64)
+
+
+_COUNTS_CACHE = {}
+
+
+def allowed_counts(w):
+    """Per-query number of allowed keys, from the oracle's own mask (cached per workload)."""
+    from oracle import clear_oracle as oracle
+    key = (w.grid_h, w.grid_w, w.n_text, w.radius)
+    if key not in _COUNTS_CACHE:
+        _COUNTS_CACHE[key] = oracle.mask_counts(w.grid_h, w.grid_w, w.n_text, w.radius)[1]
+    return _COUNTS_CACHE[key]
+
+
+def time_oracle_sample(w, q, k, v, target_s=12.0):
+    """Oracle throughput on a bounded sample of query rows of head 0, in the metric's unit:
+    4 * (allowed pairs of the sampled rows) * head_dim / seconds."""
+    from oracle import clear_oracle as oracle
+    counts = allowed_counts(w)
+    pilot = sample_rows_for_cpu(w, 2, 64)
+    t0 = time.perf_counter()
+    oracle.attn_rows(q, k, v, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale, pilot)
+    t_pilot = time.perf_counter() - t0
+    scale_up = max(1.0, target_s / max(t_pilot, 1e-3))
+    n_text_rows = max(2, int(2 * scale_up))
+    n_img_rows = max(64, int(64 * scale_up))
+    rows = sample_rows_for_cpu(w, n_text_rows, n_img_rows, seed=1)
+    t0 = time.perf_counter()
+    oracle.attn_rows(q, k, v, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale, rows)
+    dt = time.perf_counter() - t0
+    pairs = int(counts[rows[:, 2]].sum())
+    tflops = 4.0 * pairs * w.head_dim / dt / 1e12
+    return {"value": tflops, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{len(rows)} query rows of head 0 ({n_text_rows} text, {n_img_rows} image), "
+                      f"{pairs} allowed pairs, {dt:.2f} s"}, dt, pairs
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    q, k, v = workloads.make_inputs(w, heads=1)
+    per_step_target = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
+    times, pairs_all = [], []
+    info = None
+    for s in range(args.warmup + args.steps):
+        info, dt, pairs = time_oracle_sample(w, q, k, v, target_s=per_step_target)
+        if s >= args.warmup:
+            times.append(dt)
+            pairs_all.append(pairs)
+    value = 4.0 * sum(pairs_all) * w.head_dim / sum(times) / 1e12
+    info["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w), "cpu_baseline": info,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(w):
+    return {"workload": w.name, "B": w.B, "H": w.H, "head_dim": w.head_dim, "grid_h": w.grid_h, "grid_w": w.grid_w,
+            "n_text": w.n_text, "radius": w.radius, "l2": "inputs larger than L2 (no flush)" if
+            4 * w.B * w.H * w.n_tokens * w.head_dim * 2 > 126e6 * 2 else "L2 flushed between steps"}
+
+
+def run_ours(args, w):
+    from paper_2412_16112_b200 import binding as clear
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    peaks, peaks_kind = load_peaks()
+    q, k, v = workloads.make_inputs(w)
+    dtype_code = clear.BF16 if w.dtype == "bf16" else clear.F32
+    plan = clear.Plan(w.B, w.H, w.grid_h, w.grid_w, w.n_text, w.head_dim, w.radius, dtype=dtype_code)
+    info = plan.info()
+    flops = info.flops
+    qd, kd, vd = (t.to(dev) for t in (q, k, v))
+    out = torch.empty_like(qd)
+    stream = torch.cuda.current_stream()
+    small = 4 * qd.numel() * qd.element_size() <= 2 * 126e6
+    flush = torch.empty(int(256e6), dtype=torch.uint8, device=dev) if small else None
+    launches_per_call = 1 + (1 if (info.kernel == clear.KERNEL_TCGEN05 and info.n_text_splits > 1) else 0)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        plan.forward(qd, kd, vd, out, w.scale)
+    plan.check()
+
+    # ---- device-resident timing -----------------------------------------------------------------
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        t_wall0 = time.perf_counter()
+        for s in range(args.steps):
+            if flush is not None:
+                flush.fill_(s & 0xFF)
+            ev[s][0].record(stream)
+            plan.forward(qd, kd, vd, out, w.scale)
+            ev[s][1].record(stream)
+        barrier()
+        t_wall = time.perf_counter() - t_wall0
+    plan.check()
+    ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = float(sum(ms))
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    clock_info = clocks.summary()
+
+    # ---- end to end: host tensors in pinned memory, copies inside the timed region ----------------
+    e2e = None
+    if not args.no_e2e:
+        qh, kh, vh = (t.pin_memory() for t in (q, k, v))
+        oh = torch.empty_like(q).pin_memory()
+        n_e2e = max(1, min(args.steps, 5))
+        plan.forward_host(qh, kh, vh, oh, w.scale)  # allocates the staging buffers
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(n_e2e):
+            plan.forward_host(qh, kh, vh, oh, w.scale)
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / n_e2e
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        nbytes = q.numel() * q.element_size()
+        e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes, "steps": n_e2e}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant kernel ------------------------------------------------------------
+    per_gpu_tflops = flops / (ms_per_step * 1e-3) / 1e12
+    peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        try:
+            with open(tpath) as f:
+                traffic = json.load(f).get(w.name)
+        except Exception:
+            traffic = None
+    if info.kernel == clear.KERNEL_TCGEN05:
+        roofline = {"bound": "tensor", "achieved": per_gpu_tflops, "peak": peak, "unit": "TFLOP/s",
+                    "frac": per_gpu_tflops / peak, "traffic": traffic, "peak_kind": f"{peaks_kind} bf16 burst",
+                    "frac_of_sustained": per_gpu_tflops / float(peaks.get("bf16_tflops_sustained", peak)),
+                    "executed_tflops": per_gpu_tflops * info.executed_pairs / info.sum_mask,
+                    "geometric_efficiency": info.sum_mask / info.executed_pairs,
+                    "kernel": "clear_tc_kernel (+ combine kernel inside the same events)"}
+    else:
+        # fp32 CUDA-core kernel: 128 FMA lanes x 2 flops per SM per clock
+        alu_peak = 148 * 128 * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+        roofline = {"bound": "alu", "achieved": per_gpu_tflops, "peak": alu_peak, "unit": "TFLOP/s",
+                    "frac": per_gpu_tflops / alu_peak, "traffic": traffic, "peak_kind": "148 SMs x 128 fp32 FMA lanes",
+                    "kernel": "clear_simt_kernel"}
+
+    cpu_baseline = None
+    if not args.no_cpu:
+        cpu_baseline, _, _ = time_oracle_sample(w, q[:, :1].contiguous(), k[:, :1].contiguous(),
+                                                v[:, :1].contiguous())
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": workload_config(w), "clocks": clock_info, "e2e": e2e,
+            "gpu_launches": launches_per_call * args.steps, "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "ms_min": float(min(ms)), "ms_median": float(np.median(ms)), "wall_s_timed_region": t_wall,
+            "flops_per_call": flops, "sum_mask_per_head": info.sum_mask, "parallelism": "replicas"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c4_8k_r16", choices=sorted(workloads.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = workloads.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+    return run_ours(args, w)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

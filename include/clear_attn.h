@@ -1,0 +1,171 @@
+/*
+ * clear_attn.h -- C ABI of the CLEAR attention forward library for NVIDIA B200 (sm_100a).
+ *
+ * The operator (Sec. 3.2 of the CLEAR paper, arXiv 2412.16112):
+ *   tokens are [n_text text tokens ; grid_h * grid_w image tokens, row-major on the 2-D latent
+ *   grid]; the attention mask of Eq. 3 allows a (query i, key j) pair when i is a text token,
+ *   or j is a text token, or both are image tokens whose grid positions are at Euclidean
+ *   distance strictly below `radius` (window clipped at the grid border, no wrap-around);
+ *   the output is the masked softmax attention of Eq. 1,
+ *       out_i = sum_j softmax_j(scale * q_i . k_j) v_j   over the allowed j,
+ *   computed independently for every batch entry and head with the same mask.
+ *
+ * Conventions shared by every entry point
+ *   - q, k, v, out are [B, H, N, head_dim] contiguous, N = n_text + grid_h * grid_w; image token
+ *     p sits at grid row p / grid_w and column p % grid_w.
+ *   - Unless an entry point says "host", tensor pointers are DEVICE pointers on the device that
+ *     was current when the plan was created, 16-byte aligned; `out` must not overlap an input.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Forward
+ *     calls only enqueue work on it and never synchronise the host.
+ *   - Every function returns a clear_status code; nothing throws, aborts or prints.
+ *   - The library has no CPU fallback: without a usable CUDA device the calls fail with
+ *     CLEAR_ERR_CUDA.
+ */
+#ifndef CLEAR_ATTN_H_
+#define CLEAR_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum clear_status {
+    CLEAR_OK = 0,
+    CLEAR_ERR_INVALID_ARG = -1,    /* null pointer, non-positive size, radius <= 0, non-finite value */
+    CLEAR_ERR_UNSUPPORTED = -2,    /* shape or dtype outside what the requested kernel handles      */
+    CLEAR_ERR_MISALIGNED = -3,     /* a tensor pointer is not 16-byte aligned                        */
+    CLEAR_ERR_PLAN_MISMATCH = -4,  /* plan used on another device / with a kernel it was not built for */
+    CLEAR_ERR_CUDA = -5,           /* a CUDA runtime or driver call failed (see clear_last_cuda_error) */
+    CLEAR_ERR_DEVICE_TIMEOUT = -6, /* a bounded wait inside a kernel expired; outputs are invalid    */
+    CLEAR_ERR_NO_MEMORY = -7       /* host or device allocation failed                               */
+} clear_status;
+
+typedef enum clear_dtype { CLEAR_BF16 = 0, CLEAR_F32 = 1 } clear_dtype;
+
+/* Which kernel a plan drives.
+ *   AUTO    : TCGEN05 when it applies (bf16, head_dim 64 or 128, scale > 0 at call time), else SIMT.
+ *   SIMT    : exact-order fp32 CUDA-core kernel; any head_dim <= 256, bf16 or fp32 tensors.
+ *   TCGEN05 : block-sparse flash-style kernel on the 5th-generation tensor cores (TMA + TMEM). */
+typedef enum clear_kernel { CLEAR_KERNEL_AUTO = 0, CLEAR_KERNEL_SIMT = 1, CLEAR_KERNEL_TCGEN05 = 2 } clear_kernel;
+
+typedef struct clear_plan clear_plan_t; /* opaque */
+
+typedef struct clear_plan_info {
+    int32_t B, H, grid_h, grid_w, n_text, head_dim;
+    int32_t dtype;             /* clear_dtype                                                       */
+    int32_t kernel;            /* clear_kernel actually selected (never AUTO)                       */
+    int32_t radius_sq_ceil;    /* integer threshold: a pair is allowed when dx^2 + dy^2 < this      */
+    int32_t tile_h, tile_w;    /* 2-D query / key patch of the tensor-core kernel (0 for SIMT)      */
+    int32_t n_work_items;      /* work items per (batch, head)                                      */
+    int32_t n_text_splits;     /* key ranges each text-query tile is split into                     */
+    int32_t max_item_tiles;    /* longest key-tile list of any work item                            */
+    int64_t sum_mask;          /* sum(M) of Eq. 3 for one (batch, head): allowed (query, key) pairs */
+    int64_t executed_pairs;    /* (query, key) pairs the kernel's tiles cover, one (batch, head)    */
+    int64_t workspace_bytes;   /* device scratch owned by the plan                                  */
+    double flops;              /* 4 * sum_mask * head_dim * H * B  (Fig. 2 caption: 4 * sum(M) * c) */
+} clear_plan_info_t;
+
+/* ---- schedule tables (read-only views for inspection and tests) --------------------------- */
+
+/* One key/value tile of 128 keys that a work item visits. */
+typedef struct clear_kv_tile {
+    int32_t x;       /* image patch: grid column of its first key (may be negative or reach past  */
+    int32_t y;       /*   the grid: such keys are masked); linear tile: x = first token, y = 0    */
+    int32_t flags;   /* CLEAR_TILE_* bits                                                         */
+    int32_t n_valid; /* linear tile: keys [0, n_valid) of the tile exist / are allowed            */
+} clear_kv_tile_t;
+
+enum {
+    CLEAR_TILE_LINEAR = 1, /* 128 consecutive tokens of the [text; image] sequence, else a 2-D patch */
+    CLEAR_TILE_MASKED = 2  /* some (query, key) pair of the tile is not allowed: apply Eq. 3 / n_valid */
+};
+
+/* One unit of work of the tensor-core kernel: 128 queries against a list of key tiles. */
+typedef struct clear_work_item {
+    int32_t kind;         /* 0 = 2-D patch of image queries, 1 = 128 consecutive text queries      */
+    int32_t qx, qy;       /* image: grid column / row of the patch origin; text: qx = first token  */
+    int32_t n_rows;       /* queries of the tile that exist (text: min(128, n_text - qx))          */
+    int32_t tile_begin;   /* first entry of its list in the key-tile table                         */
+    int32_t tile_count;   /* length of the list (>= 1)                                             */
+    int32_t partial_slot; /* -1: writes final outputs; else index of its split-KV partial result   */
+    int32_t reserved;
+} clear_work_item_t;
+
+/* Eq. 1 under the mask of Eq. 3 for bf16 tensors, fp32 accumulation, bf16 output.
+ * A plan for the shape is looked up in (or added to) a process-wide cache, so the first call for
+ * a shape allocates and copies small tables; later calls only launch kernels.
+ * Errors: INVALID_ARG (B, H, grid_h, grid_w, head_dim <= 0; n_text < 0; radius <= 0 or
+ * non-finite; scale non-finite; null tensor), MISALIGNED, UNSUPPORTED (head_dim > 256), CUDA. */
+int clear_attn_fwd(const void *q, const void *k, const void *v, void *out, int B, int H, int grid_h,
+                   int grid_w, int n_text, int head_dim, float radius, float scale, void *stream);
+
+/* The same operator for fp32 tensors on the fp32 CUDA-core kernel (fp32 in, fp32 accumulate,
+ * fp32 out; Eq. 1 and Eq. 3 as above).  Same errors. */
+int clear_attn_fwd_f32(const void *q, const void *k, const void *v, void *out, int B, int H,
+                       int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale,
+                       void *stream);
+
+/* Build the schedule for one shape on the current device (Eq. 3 turned into integer geometry):
+ * the threshold ceil(radius^2), for every 2-D query patch the list of key patches that meet its
+ * radius-r dilation (with a flag telling whether the exact mask is needed) plus the text tiles,
+ * text-query tiles split over key ranges, and an order of the work items that evens out the load.
+ * The plan owns its device tables and workspace; the caller owns the handle and must destroy it
+ * when no call using it is still running.  `*plan` is written only on CLEAR_OK.
+ * Errors: INVALID_ARG, UNSUPPORTED (kernel/dtype/head_dim combination), CUDA, NO_MEMORY. */
+int clear_plan_create(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text,
+                      int head_dim, float radius, int dtype, int kernel);
+
+/* The same schedule built on the host only: no CUDA call is made and no device is needed.  The
+ * plan can be inspected (clear_plan_info, clear_plan_tables) and destroyed, not executed
+ * (forward calls return PLAN_MISMATCH).  Errors: INVALID_ARG, UNSUPPORTED, NO_MEMORY. */
+int clear_plan_create_host(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text,
+                           int head_dim, float radius, int dtype, int kernel);
+
+/* Borrow the host copies of the schedule tables (valid until the plan is destroyed).  Any output
+ * pointer may be NULL.  `half_width[dy]`, dy in [0, n_half_width), is the largest |dx| allowed at
+ * row offset dy.  For SIMT plans the item and tile tables are empty.  Errors: INVALID_ARG. */
+int clear_plan_tables(const clear_plan_t *plan, const clear_work_item_t **items, int32_t *n_items,
+                      const clear_kv_tile_t **tiles, int32_t *n_tiles, const int32_t **half_width,
+                      int32_t *n_half_width);
+
+/* Forward pass with an explicit plan.  Tensor dtype is the plan's.  Calls on one plan share its
+ * workspace: run them on one stream, or order them yourself.
+ * Errors: INVALID_ARG, MISALIGNED, PLAN_MISMATCH (current device differs from the plan's),
+ * UNSUPPORTED (tensor-core plan called with scale <= 0), CUDA. */
+int clear_attn_fwd_planned(const clear_plan_t *plan, const void *q, const void *k, const void *v,
+                           void *out, float scale, void *stream);
+
+/* Forward pass on HOST tensors (same layout and dtype as the plan's): copies q, k, v to staging
+ * buffers the plan owns (allocated on first use), runs the kernels, copies `out` back, all on
+ * `stream`, and returns after synchronising that stream.  Pinned host memory makes the copies
+ * asynchronous with respect to other streams.  Errors as clear_attn_fwd_planned, plus NO_MEMORY
+ * and DEVICE_TIMEOUT. */
+int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_host,
+                        const void *v_host, void *out_host, float scale, void *stream);
+
+/* Fill `info` from the plan (host only, no CUDA call).  Errors: INVALID_ARG. */
+int clear_plan_info(const clear_plan_t *plan, clear_plan_info_t *info);
+
+/* Synchronise `stream`, then read and clear the plan's device status word.  Returns
+ * CLEAR_ERR_DEVICE_TIMEOUT if any kernel launched with this plan gave up on a bounded wait since
+ * the last check, CLEAR_OK otherwise.  Errors: INVALID_ARG, CUDA. */
+int clear_plan_check(clear_plan_t *plan, void *stream);
+
+/* Free the plan's device memory and the handle.  NULL is accepted.  Errors: CUDA. */
+int clear_plan_destroy(clear_plan_t *plan);
+
+/* Drop every plan the unplanned entry points cached (synchronises the device first). */
+int clear_cache_clear(void);
+
+/* Static, human-readable name of a status code. */
+const char *clear_status_string(int status);
+
+/* cudaError_t value of the most recent CUDA failure seen by the calling thread (0 if none). */
+int clear_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CLEAR_ATTN_H_ */

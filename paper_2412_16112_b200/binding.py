@@ -1,0 +1,213 @@
+"""ctypes binding of ``libclear_attn.so``: same names as the C ABI, argument marshalling only.
+
+Every step of the attention path runs in the library's CUDA kernels; PyTorch appears here only
+as the owner of device memory and streams (``data_ptr()``, ``current_stream()``).  There is no
+fallback: if the library cannot be loaded, or a call fails, a ``ClearError`` is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+from typing import Optional
+
+from . import build as _build
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_PLAN_MISMATCH = -1, -2, -3, -4
+ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY = -5, -6, -7
+BF16, F32 = 0, 1
+KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05 = 0, 1, 2
+TILE_LINEAR, TILE_MASKED = 1, 2
+
+EXPORTS = [
+    "clear_attn_fwd", "clear_attn_fwd_f32", "clear_plan_create", "clear_plan_create_host",
+    "clear_plan_tables", "clear_attn_fwd_planned", "clear_attn_fwd_host", "clear_plan_info",
+    "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
+    "clear_last_cuda_error",
+]
+
+
+class ClearError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} (status {status}, cuda error {last_cuda_error()})")
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("B", "H", "grid_h", "grid_w", "n_text", "head_dim", "dtype", "kernel", "radius_sq_ceil",
+                 "tile_h", "tile_w", "n_work_items", "n_text_splits", "max_item_tiles")] + \
+               [("sum_mask", ctypes.c_int64), ("executed_pairs", ctypes.c_int64),
+                ("workspace_bytes", ctypes.c_int64), ("flops", ctypes.c_double)]
+
+
+class KvTile(ctypes.Structure):
+    _fields_ = [("x", ctypes.c_int32), ("y", ctypes.c_int32), ("flags", ctypes.c_int32),
+                ("n_valid", ctypes.c_int32)]
+
+
+class WorkItem(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("kind", "qx", "qy", "n_rows", "tile_begin", "tile_count", "partial_slot", "reserved")]
+
+
+_lock = threading.Lock()
+_lib: Optional[ctypes.CDLL] = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load() -> ctypes.CDLL:
+    """Load the shared library (building it with nvcc first if it is missing or stale)."""
+    global _lib
+    with _lock:
+        if _lib is not None:
+            return _lib
+        path = _build.LIB
+        if not os.path.exists(path) or os.environ.get("CLEAR_REBUILD") == "1":
+            path = _build.build()
+        lib = ctypes.CDLL(path)
+        vp, i32, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+        fwd_args = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp]
+        lib.clear_attn_fwd.argtypes = fwd_args
+        lib.clear_attn_fwd_f32.argtypes = fwd_args
+        plan_args = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, f32, i32, i32]
+        lib.clear_plan_create.argtypes = plan_args
+        lib.clear_plan_create_host.argtypes = plan_args
+        lib.clear_plan_tables.argtypes = [vp, ctypes.POINTER(ctypes.POINTER(WorkItem)), ctypes.POINTER(ctypes.c_int32),
+                                          ctypes.POINTER(ctypes.POINTER(KvTile)), ctypes.POINTER(ctypes.c_int32),
+                                          ctypes.POINTER(ctypes.POINTER(ctypes.c_int32)),
+                                          ctypes.POINTER(ctypes.c_int32)]
+        lib.clear_attn_fwd_planned.argtypes = [vp, vp, vp, vp, vp, f32, vp]
+        lib.clear_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, f32, vp]
+        lib.clear_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
+        lib.clear_plan_check.argtypes = [vp, vp]
+        lib.clear_plan_destroy.argtypes = [vp]
+        lib.clear_cache_clear.argtypes = []
+        lib.clear_status_string.argtypes = [i32]
+        lib.clear_status_string.restype = ctypes.c_char_p
+        lib.clear_last_cuda_error.argtypes = []
+        for name in EXPORTS:
+            if name != "clear_status_string":
+                getattr(lib, name).restype = i32
+        _lib = lib
+        return lib
+
+
+def status_string(status: int) -> str:
+    return load().clear_status_string(int(status)).decode()
+
+
+def last_cuda_error() -> int:
+    return int(load().clear_last_cuda_error())
+
+
+def _check(status: int, what: str) -> None:
+    if status != OK:
+        raise ClearError(status, what)
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _tensor_args(q, k, v, out, dtype_code):
+    import torch
+    want = torch.bfloat16 if dtype_code == BF16 else torch.float32
+    for name, t in (("q", q), ("k", k), ("v", v), ("out", out)):
+        if not t.is_cuda:
+            raise ValueError(f"{name} must be a CUDA tensor")
+        if t.dtype != want:
+            raise TypeError(f"{name} must be {want}")
+        if not t.is_contiguous():
+            raise ValueError(f"{name} must be contiguous [B, H, N, d]")
+    if not (q.shape == k.shape == v.shape == out.shape) or q.dim() != 4:
+        raise ValueError("q, k, v, out must share one [B, H, N, d] shape")
+    return q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()
+
+
+def clear_attn_fwd(q, k, v, out, grid_h, grid_w, n_text, radius, scale, stream=None):
+    """bf16 CLEAR attention forward into ``out``; tensors are [B, H, n_text + grid_h*grid_w, d]."""
+    ptrs = _tensor_args(q, k, v, out, BF16)
+    B, H, _, d = q.shape
+    _check(load().clear_attn_fwd(*ptrs, B, H, grid_h, grid_w, n_text, d, float(radius), float(scale),
+                                 _stream_ptr(stream)), "clear_attn_fwd")
+    return out
+
+
+def clear_attn_fwd_f32(q, k, v, out, grid_h, grid_w, n_text, radius, scale, stream=None):
+    """fp32 CLEAR attention forward into ``out``."""
+    ptrs = _tensor_args(q, k, v, out, F32)
+    B, H, _, d = q.shape
+    _check(load().clear_attn_fwd_f32(*ptrs, B, H, grid_h, grid_w, n_text, d, float(radius), float(scale),
+                                     _stream_ptr(stream)), "clear_attn_fwd_f32")
+    return out
+
+
+class Plan:
+    """Owner of a ``clear_plan_t``."""
+
+    def __init__(self, B, H, grid_h, grid_w, n_text, head_dim, radius, dtype=BF16, kernel=KERNEL_AUTO,
+                 host_only=False):
+        self._h = ctypes.c_void_p()
+        fn = load().clear_plan_create_host if host_only else load().clear_plan_create
+        _check(fn(ctypes.byref(self._h), B, H, grid_h, grid_w, n_text, head_dim, float(radius), dtype, kernel),
+               "clear_plan_create_host" if host_only else "clear_plan_create")
+        self.dtype = dtype
+
+    @property
+    def handle(self):
+        return self._h
+
+    def info(self) -> PlanInfo:
+        out = PlanInfo()
+        _check(load().clear_plan_info(self._h, ctypes.byref(out)), "clear_plan_info")
+        return out
+
+    def tables(self):
+        """(items, tiles, half_width) as lists of ctypes structs / ints (copies)."""
+        items, tiles, hw = ctypes.POINTER(WorkItem)(), ctypes.POINTER(KvTile)(), ctypes.POINTER(ctypes.c_int32)()
+        ni, nt, nh = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+        _check(load().clear_plan_tables(self._h, ctypes.byref(items), ctypes.byref(ni), ctypes.byref(tiles),
+                                        ctypes.byref(nt), ctypes.byref(hw), ctypes.byref(nh)), "clear_plan_tables")
+        return ([items[i] for i in range(ni.value)], [tiles[i] for i in range(nt.value)],
+                [hw[i] for i in range(nh.value)])
+
+    def forward(self, q, k, v, out, scale, stream=None):
+        ptrs = _tensor_args(q, k, v, out, self.dtype)
+        _check(load().clear_attn_fwd_planned(self._h, *ptrs, float(scale), _stream_ptr(stream)),
+               "clear_attn_fwd_planned")
+        return out
+
+    def forward_host(self, q, k, v, out, scale, stream=None):
+        """Host (CPU, ideally pinned) tensors in, host tensor out; returns after the stream is idle."""
+        for t in (q, k, v, out):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("forward_host takes contiguous CPU tensors")
+        _check(load().clear_attn_fwd_host(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                          float(scale), _stream_ptr(stream)), "clear_attn_fwd_host")
+        return out
+
+    def check(self, stream=None) -> None:
+        _check(load().clear_plan_check(self._h, _stream_ptr(stream)), "clear_plan_check")
+
+    def destroy(self) -> None:
+        if self._h:
+            load().clear_plan_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def clear_cache_clear() -> None:
+    _check(load().clear_cache_clear(), "clear_cache_clear")

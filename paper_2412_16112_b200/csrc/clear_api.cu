@@ -1,0 +1,367 @@
+// C ABI of the CLEAR attention library: argument checks, plans, plan cache, launches.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <list>
+#include <memory>
+#include <new>
+
+#include "clear_internal.hpp"
+
+namespace clear {
+
+static thread_local int g_last_cuda_error = 0;
+void note_cuda_error(int err) { g_last_cuda_error = err; }
+
+namespace {
+
+int select_kernel(const Shape &s)
+{
+    if (s.kernel != CLEAR_KERNEL_AUTO) return s.kernel;
+    if (s.dtype == CLEAR_BF16 && (s.head_dim == 64 || s.head_dim == 128)) return CLEAR_KERNEL_TCGEN05;
+    return CLEAR_KERNEL_SIMT;
+}
+
+template <typename T>
+int upload(T **dst, const std::vector<T> &src)
+{
+    *dst = nullptr;
+    if (src.empty()) return CLEAR_OK;
+    CLEAR_CUDA_TRY(cudaMalloc((void **)dst, src.size() * sizeof(T)));
+    CLEAR_CUDA_TRY(cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice));
+    return CLEAR_OK;
+}
+
+int free_device_parts(clear_plan *p)
+{
+    int rc = CLEAR_OK;
+    auto rel = [&](void *ptr) {
+        if (ptr && cudaFree(ptr) != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = CLEAR_ERR_CUDA;
+        }
+    };
+    rel(p->d_half_width);
+    rel(p->d_items);
+    rel(p->d_tiles);
+    rel(p->d_status);
+    rel(p->d_partial_o);
+    rel(p->d_partial_ml);
+    for (void *&s : p->d_stage) {
+        rel(s);
+        s = nullptr;
+    }
+    p->d_half_width = nullptr;
+    p->d_items = nullptr;
+    p->d_tiles = nullptr;
+    p->d_status = nullptr;
+    p->d_partial_o = nullptr;
+    p->d_partial_ml = nullptr;
+    return rc;
+}
+
+int create_plan(clear_plan_t **out, const Shape &shape_in, bool host_only)
+{
+    if (!out) return CLEAR_ERR_INVALID_ARG;
+    Shape s = shape_in;
+    int rc = validate_shape(s);
+    if (rc != CLEAR_OK) return rc;
+    const int kernel = select_kernel(s);
+    {
+        Shape chk = s;
+        chk.kernel = kernel;
+        rc = validate_shape(chk);
+        if (rc != CLEAR_OK) return rc;
+    }
+    std::unique_ptr<clear_plan> p(new (std::nothrow) clear_plan());
+    if (!p) return CLEAR_ERR_NO_MEMORY;
+    p->shape = s;
+    p->kernel = kernel;
+    p->host_only = host_only;
+    try {
+        if (kernel == CLEAR_KERNEL_TCGEN05)
+            build_tile_schedule(s, p->sch);
+        else
+            build_geometry(s, p->sch);
+    } catch (const std::bad_alloc &) {
+        return CLEAR_ERR_NO_MEMORY;
+    }
+    if (kernel == CLEAR_KERNEL_TCGEN05 && p->sch.n_partial_slots > 0) {
+        const int64_t rows = (int64_t)s.B * s.H * p->sch.n_partial_slots * kTileTokens;
+        p->workspace_bytes = rows * (s.head_dim + 2) * (int64_t)sizeof(float);
+    }
+    if (!host_only) {
+        CLEAR_CUDA_TRY(cudaGetDevice(&p->device));
+        rc = upload(&p->d_half_width, p->sch.half_width);
+        if (rc == CLEAR_OK) rc = upload(&p->d_items, p->sch.items);
+        if (rc == CLEAR_OK) rc = upload(&p->d_tiles, p->sch.tiles);
+        if (rc == CLEAR_OK) {
+            cudaError_t e = cudaMalloc((void **)&p->d_status, sizeof(int));
+            if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
+            if (e != cudaSuccess) {
+                note_cuda_error((int)e);
+                (void)cudaGetLastError();
+                rc = CLEAR_ERR_CUDA;
+            }
+        }
+        if (rc == CLEAR_OK && p->workspace_bytes > 0) {
+            const int64_t rows = (int64_t)s.B * s.H * p->sch.n_partial_slots * kTileTokens;
+            cudaError_t e = cudaMalloc((void **)&p->d_partial_o, (size_t)rows * s.head_dim * sizeof(float));
+            if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_partial_ml, (size_t)rows * 2 * sizeof(float));
+            if (e != cudaSuccess) {
+                note_cuda_error((int)e);
+                (void)cudaGetLastError();
+                rc = e == cudaErrorMemoryAllocation ? CLEAR_ERR_NO_MEMORY : CLEAR_ERR_CUDA;
+            }
+        }
+        if (rc != CLEAR_OK) {
+            free_device_parts(p.get());
+            return rc;
+        }
+    }
+    *out = p.release();
+    return CLEAR_OK;
+}
+
+int check_tensors(const void *q, const void *k, const void *v, const void *out)
+{
+    if (!q || !k || !v || !out) return CLEAR_ERR_INVALID_ARG;
+    const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out;
+    if (bits & 15u) return CLEAR_ERR_MISALIGNED;
+    return CLEAR_OK;
+}
+
+int forward(const clear_plan *p, const void *q, const void *k, const void *v, void *out, float scale, void *stream)
+{
+    if (!p) return CLEAR_ERR_INVALID_ARG;
+    if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
+    int rc = check_tensors(q, k, v, out);
+    if (rc != CLEAR_OK) return rc;
+    if (p->host_only) return CLEAR_ERR_PLAN_MISMATCH;
+    int dev = -1;
+    CLEAR_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != p->device) return CLEAR_ERR_PLAN_MISMATCH;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (p->kernel == CLEAR_KERNEL_TCGEN05) return launch_tc(*p, q, k, v, out, scale, st);
+    return launch_simt(*p, q, k, v, out, scale, st);
+}
+
+// ---- plan cache of the unplanned entry points ----------------------------------------------------
+struct CacheEntry {
+    Shape shape;
+    int device;
+    clear_plan_t *plan;
+};
+std::mutex g_cache_mutex;
+std::list<CacheEntry> g_cache;
+
+int cached_forward(const void *q, const void *k, const void *v, void *out, const Shape &shape, float scale, void *stream)
+{
+    int rc = validate_shape(shape);
+    if (rc != CLEAR_OK) return rc;
+    if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
+    rc = check_tensors(q, k, v, out);
+    if (rc != CLEAR_OK) return rc;
+    int dev = -1;
+    CLEAR_CUDA_TRY(cudaGetDevice(&dev));
+    Shape s = shape;
+    // the tensor-core kernel needs a positive scale; anything else goes to the CUDA-core kernel
+    if (s.kernel == CLEAR_KERNEL_AUTO && !(scale > 0.f)) s.kernel = CLEAR_KERNEL_SIMT;
+    clear_plan_t *plan = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_cache_mutex);
+        for (const CacheEntry &e : g_cache)
+            if (e.device == dev && e.shape == s) {
+                plan = e.plan;
+                break;
+            }
+        if (!plan) {
+            rc = create_plan(&plan, s, false);
+            if (rc != CLEAR_OK) return rc;
+            g_cache.push_front(CacheEntry{s, dev, plan});
+        }
+    }
+    return forward(plan, q, k, v, out, scale, stream);
+}
+
+}  // namespace
+}  // namespace clear
+
+using namespace clear;
+
+extern "C" {
+
+int clear_attn_fwd(const void *q, const void *k, const void *v, void *out, int B, int H, int grid_h, int grid_w,
+                   int n_text, int head_dim, float radius, float scale, void *stream)
+{
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, CLEAR_BF16, CLEAR_KERNEL_AUTO};
+    return cached_forward(q, k, v, out, s, scale, stream);
+}
+
+int clear_attn_fwd_f32(const void *q, const void *k, const void *v, void *out, int B, int H, int grid_h, int grid_w,
+                       int n_text, int head_dim, float radius, float scale, void *stream)
+{
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, CLEAR_F32, CLEAR_KERNEL_SIMT};
+    return cached_forward(q, k, v, out, s, scale, stream);
+}
+
+int clear_plan_create(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text, int head_dim,
+                      float radius, int dtype, int kernel)
+{
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, dtype, kernel};
+    return create_plan(plan, s, false);
+}
+
+int clear_plan_create_host(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text, int head_dim,
+                           float radius, int dtype, int kernel)
+{
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, dtype, kernel};
+    return create_plan(plan, s, true);
+}
+
+int clear_plan_tables(const clear_plan_t *plan, const clear_work_item_t **items, int32_t *n_items,
+                      const clear_kv_tile_t **tiles, int32_t *n_tiles, const int32_t **half_width,
+                      int32_t *n_half_width)
+{
+    if (!plan) return CLEAR_ERR_INVALID_ARG;
+    if (items) *items = plan->sch.items.data();
+    if (n_items) *n_items = (int32_t)plan->sch.items.size();
+    if (tiles) *tiles = plan->sch.tiles.data();
+    if (n_tiles) *n_tiles = (int32_t)plan->sch.tiles.size();
+    if (half_width) *half_width = plan->sch.half_width.data();
+    if (n_half_width) *n_half_width = (int32_t)plan->sch.half_width.size();
+    return CLEAR_OK;
+}
+
+int clear_attn_fwd_planned(const clear_plan_t *plan, const void *q, const void *k, const void *v, void *out,
+                           float scale, void *stream)
+{
+    return forward(plan, q, k, v, out, scale, stream);
+}
+
+int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_host, const void *v_host,
+                        void *out_host, float scale, void *stream)
+{
+    if (!plan || !q_host || !k_host || !v_host || !out_host) return CLEAR_ERR_INVALID_ARG;
+    if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
+    if (plan->host_only) return CLEAR_ERR_PLAN_MISMATCH;
+    int dev = -1;
+    CLEAR_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != plan->device) return CLEAR_ERR_PLAN_MISMATCH;
+    const Shape &s = plan->shape;
+    const size_t esz = s.dtype == CLEAR_BF16 ? 2 : 4;
+    const size_t bytes = (size_t)s.B * s.H * ((size_t)s.n_text + (size_t)s.grid_h * s.grid_w) * s.head_dim * esz;
+    for (void *&st : plan->d_stage) {
+        if (!st) {
+            cudaError_t e = cudaMalloc(&st, bytes);
+            if (e != cudaSuccess) {
+                st = nullptr;
+                note_cuda_error((int)e);
+                (void)cudaGetLastError();
+                return e == cudaErrorMemoryAllocation ? CLEAR_ERR_NO_MEMORY : CLEAR_ERR_CUDA;
+            }
+        }
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[0], q_host, bytes, cudaMemcpyHostToDevice, cs));
+    CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[1], k_host, bytes, cudaMemcpyHostToDevice, cs));
+    CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[2], v_host, bytes, cudaMemcpyHostToDevice, cs));
+    int rc = forward(plan, plan->d_stage[0], plan->d_stage[1], plan->d_stage[2], plan->d_stage[3], scale, stream);
+    if (rc != CLEAR_OK) return rc;
+    CLEAR_CUDA_TRY(cudaMemcpyAsync(out_host, plan->d_stage[3], bytes, cudaMemcpyDeviceToHost, cs));
+    return clear_plan_check(plan, stream);
+}
+
+int clear_plan_info(const clear_plan_t *plan, clear_plan_info_t *info)
+{
+    if (!plan || !info) return CLEAR_ERR_INVALID_ARG;
+    const Shape &s = plan->shape;
+    std::memset(info, 0, sizeof(*info));
+    info->B = s.B;
+    info->H = s.H;
+    info->grid_h = s.grid_h;
+    info->grid_w = s.grid_w;
+    info->n_text = s.n_text;
+    info->head_dim = s.head_dim;
+    info->dtype = s.dtype;
+    info->kernel = plan->kernel;
+    info->radius_sq_ceil = (int32_t)plan->sch.thr;
+    const bool tc = plan->kernel == CLEAR_KERNEL_TCGEN05;
+    info->tile_h = tc ? kTileH : 0;
+    info->tile_w = tc ? kTileW : 0;
+    info->n_work_items = (int32_t)plan->sch.items.size();
+    info->n_text_splits = plan->sch.n_text_splits;
+    info->max_item_tiles = plan->sch.max_item_tiles;
+    info->sum_mask = plan->sch.sum_mask;
+    info->executed_pairs = tc ? plan->sch.executed_pairs : plan->sch.sum_mask;
+    info->workspace_bytes = plan->workspace_bytes;
+    info->flops = 4.0 * (double)plan->sch.sum_mask * s.head_dim * s.H * s.B;
+    return CLEAR_OK;
+}
+
+int clear_plan_check(clear_plan_t *plan, void *stream)
+{
+    if (!plan) return CLEAR_ERR_INVALID_ARG;
+    if (plan->host_only) return CLEAR_ERR_PLAN_MISMATCH;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    int status = 0;
+    CLEAR_CUDA_TRY(cudaMemcpyAsync(&status, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost, cs));
+    CLEAR_CUDA_TRY(cudaStreamSynchronize(cs));
+    if (status != 0) {
+        CLEAR_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(int), cs));
+        CLEAR_CUDA_TRY(cudaStreamSynchronize(cs));
+        return CLEAR_ERR_DEVICE_TIMEOUT;
+    }
+    return CLEAR_OK;
+}
+
+int clear_plan_destroy(clear_plan_t *plan)
+{
+    if (!plan) return CLEAR_OK;
+    int rc = CLEAR_OK;
+    if (!plan->host_only) {
+        int prev = -1;
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != plan->device) (void)cudaSetDevice(plan->device);
+        rc = free_device_parts(plan);
+        if (prev >= 0 && prev != plan->device) (void)cudaSetDevice(prev);
+    }
+    delete plan;
+    return rc;
+}
+
+int clear_cache_clear(void)
+{
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    int rc = CLEAR_OK;
+    if (!g_cache.empty()) {
+        if (cudaDeviceSynchronize() != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = CLEAR_ERR_CUDA;
+        }
+    }
+    for (CacheEntry &e : g_cache) {
+        int r = clear_plan_destroy(e.plan);
+        if (r != CLEAR_OK) rc = r;
+    }
+    g_cache.clear();
+    return rc;
+}
+
+const char *clear_status_string(int status)
+{
+    switch (status) {
+        case CLEAR_OK: return "ok";
+        case CLEAR_ERR_INVALID_ARG: return "invalid argument";
+        case CLEAR_ERR_UNSUPPORTED: return "unsupported shape, dtype or kernel";
+        case CLEAR_ERR_MISALIGNED: return "tensor pointer is not 16-byte aligned";
+        case CLEAR_ERR_PLAN_MISMATCH: return "plan does not match this call (device, host-only plan)";
+        case CLEAR_ERR_CUDA: return "CUDA call failed";
+        case CLEAR_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case CLEAR_ERR_NO_MEMORY: return "out of memory";
+        default: return "unknown status";
+    }
+}
+
+int clear_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

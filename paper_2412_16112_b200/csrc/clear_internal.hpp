@@ -1,0 +1,60 @@
+// Internal plan object and kernel launchers shared by the C-ABI layer and the kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "clear_attn.h"
+#include "clear_plan.hpp"
+
+struct clear_plan {
+    clear::Shape shape;
+    clear::Schedule sch;
+    int kernel = CLEAR_KERNEL_SIMT;  // selected kernel (never AUTO)
+    bool host_only = false;
+    int device = -1;
+
+    // device tables (owned)
+    int32_t *d_half_width = nullptr;
+    clear_work_item_t *d_items = nullptr;
+    clear_kv_tile_t *d_tiles = nullptr;
+    int *d_status = nullptr;  // 0 = fine; set by a kernel whose bounded wait expired
+
+    // split-KV workspace of the text-query rows (owned): per (bh, slot) 128 x head_dim fp32
+    // un-normalised outputs, and per row the running maximum (log2 units) and the row sum
+    float *d_partial_o = nullptr;
+    float *d_partial_ml = nullptr;
+    int64_t workspace_bytes = 0;
+
+    // staging buffers of the host-tensor entry point (owned, allocated on first use)
+    void *d_stage[4] = {nullptr, nullptr, nullptr, nullptr};
+
+    // tensor maps of the last (q, k, v, out) seen by the tensor-core launcher
+    mutable std::mutex tm_mutex;
+    mutable const void *tm_ptrs[4] = {nullptr, nullptr, nullptr, nullptr};
+    alignas(64) mutable unsigned char tm_storage[8][128];
+    mutable bool tm_valid = false;
+};
+
+namespace clear {
+
+// Thread-local record of the last failing CUDA call.
+void note_cuda_error(int err);
+
+#define CLEAR_CUDA_TRY(expr)                          \
+    do {                                              \
+        cudaError_t _e = (expr);                      \
+        if (_e != cudaSuccess) {                      \
+            clear::note_cuda_error((int)_e);          \
+            (void)cudaGetLastError();                 \
+            return CLEAR_ERR_CUDA;                    \
+        }                                             \
+    } while (0)
+
+int launch_simt(const clear_plan &p, const void *q, const void *k, const void *v, void *out, float scale,
+                cudaStream_t stream);
+int launch_tc(const clear_plan &p, const void *q, const void *k, const void *v, void *out, float scale,
+              cudaStream_t stream);
+
+}  // namespace clear

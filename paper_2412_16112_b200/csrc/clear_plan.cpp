@@ -1,0 +1,169 @@
+// Host-side schedule of the CLEAR attention kernels: Eq. 3 turned into integer geometry,
+// the 2-D tile-pair lists, the split of the text-query rows and the work order.
+#include "clear_plan.hpp"
+
+#include <algorithm>
+#include <cmath>
+
+namespace clear {
+
+static int64_t isqrt64(int64_t v)
+{
+    if (v <= 0) return 0;
+    int64_t r = (int64_t)std::sqrt((double)v);
+    while (r * r > v) --r;
+    while ((r + 1) * (r + 1) <= v) ++r;
+    return r;
+}
+
+int validate_shape(const Shape &s)
+{
+    if (s.B <= 0 || s.H <= 0 || s.grid_h <= 0 || s.grid_w <= 0 || s.n_text < 0 || s.head_dim <= 0)
+        return CLEAR_ERR_INVALID_ARG;
+    if (!(s.radius > 0.f) || !std::isfinite(s.radius)) return CLEAR_ERR_INVALID_ARG;
+    if (s.dtype != CLEAR_BF16 && s.dtype != CLEAR_F32) return CLEAR_ERR_INVALID_ARG;
+    if (s.kernel < CLEAR_KERNEL_AUTO || s.kernel > CLEAR_KERNEL_TCGEN05) return CLEAR_ERR_INVALID_ARG;
+    const int64_t n = (int64_t)s.grid_h * s.grid_w;
+    const int64_t N = n + s.n_text;
+    if (N > (int64_t)1 << 30) return CLEAR_ERR_UNSUPPORTED;  // token indices stay in int32
+    if ((int64_t)s.B * s.H > 65535) return CLEAR_ERR_UNSUPPORTED;  // (batch, head) is a grid's y axis
+    if (s.head_dim > 256) return CLEAR_ERR_UNSUPPORTED;
+    // 16-byte rows keep every per-token vector access and TMA stride aligned
+    const int esz = s.dtype == CLEAR_BF16 ? 2 : 4;
+    if ((s.head_dim * esz) % 16 != 0) return CLEAR_ERR_UNSUPPORTED;
+    if (s.kernel == CLEAR_KERNEL_TCGEN05) {
+        if (s.dtype != CLEAR_BF16) return CLEAR_ERR_UNSUPPORTED;
+        if (s.head_dim != 64 && s.head_dim != 128) return CLEAR_ERR_UNSUPPORTED;
+    }
+    return CLEAR_OK;
+}
+
+void build_geometry(const Shape &s, Schedule &sch)
+{
+    const int64_t gh = s.grid_h, gw = s.grid_w, T = s.n_text;
+    const int64_t n = gh * gw, N = n + T;
+    // Eq. 3 with integer squared distances: d2 < r^2  <=>  d2 < ceil(r^2).  No pair on the grid
+    // is farther apart than its diagonal, so the threshold is capped just above it.
+    const double r = (double)s.radius;
+    const double r2 = std::ceil(r * r);
+    const int64_t diag2 = (gh - 1) * (gh - 1) + (gw - 1) * (gw - 1);
+    sch.thr = (r2 > (double)(diag2 + 1)) ? diag2 + 1 : (int64_t)r2;
+
+    const int64_t R = std::min<int64_t>(isqrt64(sch.thr - 1), gh - 1);  // largest |dy| that still has keys
+    sch.half_width.assign((size_t)R + 1, 0);
+    int64_t img_img = 0;
+    for (int64_t dy = 0; dy <= R; ++dy) {
+        const int64_t m = std::min<int64_t>(isqrt64(sch.thr - 1 - dy * dy), gw - 1);
+        sch.half_width[(size_t)dy] = (int32_t)m;
+        // keys in row y+dy seen by the gw queries of row y: sum_x (min(x+m, gw-1) - max(x-m, 0) + 1)
+        const int64_t row_pairs = gw * (2 * m + 1) - m * (m + 1);
+        const int64_t rows = gh - dy;  // query rows y for which y + dy is on the grid
+        img_img += (dy == 0 ? 1 : 2) * rows * row_pairs;
+    }
+    sch.sum_mask = T * N + n * T + img_img;
+}
+
+void build_tile_schedule(const Shape &s, Schedule &sch)
+{
+    build_geometry(s, sch);
+    const int gh = s.grid_h, gw = s.grid_w, T = s.n_text;
+    const int64_t N = (int64_t)gh * gw + T;
+    const int64_t thr = sch.thr;
+    const int R = (int)isqrt64(thr - 1);
+
+    sch.items.clear();
+    sch.tiles.clear();
+
+    // ---- text-query tiles: dense over all N keys, split over key ranges ------------------------
+    const int n_lin = (int)((N + kTileTokens - 1) / kTileTokens);
+    sch.n_text_tiles = (T + kTileTokens - 1) / kTileTokens;
+    int chunk = n_lin, n_splits = 1;
+    if (sch.n_text_tiles > 0) {
+        n_splits = (n_lin + kSplitTargetTiles - 1) / kSplitTargetTiles;
+        chunk = (n_lin + n_splits - 1) / n_splits;
+        n_splits = (n_lin + chunk - 1) / chunk;
+    }
+    sch.n_text_splits = sch.n_text_tiles > 0 ? n_splits : 0;
+    sch.n_partial_slots = (sch.n_text_tiles > 0 && n_splits > 1) ? sch.n_text_tiles * n_splits : 0;
+    for (int tq = 0; tq < sch.n_text_tiles; ++tq) {
+        for (int sp = 0; sp < n_splits; ++sp) {
+            clear_work_item_t it{};
+            it.kind = 1;
+            it.qx = tq * kTileTokens;
+            it.qy = 0;
+            it.n_rows = std::min(kTileTokens, T - it.qx);
+            it.tile_begin = (int32_t)sch.tiles.size();
+            const int t0 = sp * chunk, t1 = std::min(n_lin, t0 + chunk);
+            for (int t = t0; t < t1; ++t) {
+                clear_kv_tile_t kt{};
+                kt.x = t * kTileTokens;
+                kt.y = 0;
+                kt.n_valid = (int32_t)std::min<int64_t>(kTileTokens, N - (int64_t)kt.x);
+                kt.flags = CLEAR_TILE_LINEAR | (kt.n_valid < kTileTokens ? CLEAR_TILE_MASKED : 0);
+                sch.tiles.push_back(kt);
+            }
+            it.tile_count = t1 - t0;
+            it.partial_slot = n_splits > 1 ? tq * n_splits + sp : -1;
+            sch.items.push_back(it);
+        }
+    }
+
+    // ---- image-query patches: text tiles, then the key patches that meet the dilated patch -----
+    const int ntx = (gw + kTileW - 1) / kTileW, nty = (gh + kTileH - 1) / kTileH;
+    const int reach_x = R / kTileW + 1, reach_y = R / kTileH + 1;
+    for (int ty = 0; ty < nty; ++ty) {
+        for (int tx = 0; tx < ntx; ++tx) {
+            clear_work_item_t it{};
+            it.kind = 0;
+            it.qx = tx * kTileW;
+            it.qy = ty * kTileH;
+            const int qx1 = std::min(it.qx + kTileW - 1, gw - 1), qy1 = std::min(it.qy + kTileH - 1, gh - 1);
+            it.n_rows = (qx1 - it.qx + 1) * (qy1 - it.qy + 1);
+            it.tile_begin = (int32_t)sch.tiles.size();
+            for (int t0 = 0; t0 < T; t0 += kTileTokens) {
+                clear_kv_tile_t kt{};
+                kt.x = t0;
+                kt.y = 0;
+                kt.n_valid = std::min(kTileTokens, T - t0);  // tokens past n_text are image keys: not allowed here
+                kt.flags = CLEAR_TILE_LINEAR | (kt.n_valid < kTileTokens ? CLEAR_TILE_MASKED : 0);
+                sch.tiles.push_back(kt);
+            }
+            for (int j = std::max(0, ty - reach_y); j <= std::min(nty - 1, ty + reach_y); ++j) {
+                for (int i = std::max(0, tx - reach_x); i <= std::min(ntx - 1, tx + reach_x); ++i) {
+                    const int bx = i * kTileW, by = j * kTileH;
+                    const int kx1 = std::min(bx + kTileW - 1, gw - 1), ky1 = std::min(by + kTileH - 1, gh - 1);
+                    // smallest and largest coordinate differences between the two (clipped) patches
+                    const int64_t gx = std::max({0, bx - qx1, it.qx - kx1});
+                    const int64_t gy = std::max({0, by - qy1, it.qy - ky1});
+                    if (gx * gx + gy * gy >= thr) continue;
+                    const int64_t fx = std::max(kx1 - it.qx, qx1 - bx);
+                    const int64_t fy = std::max(ky1 - it.qy, qy1 - by);
+                    const bool whole = (bx + kTileW <= gw) && (by + kTileH <= gh);
+                    clear_kv_tile_t kt{};
+                    kt.x = bx;
+                    kt.y = by;
+                    kt.n_valid = kTileTokens;
+                    kt.flags = (whole && fx * fx + fy * fy < thr) ? 0 : CLEAR_TILE_MASKED;
+                    sch.tiles.push_back(kt);
+                }
+            }
+            it.tile_count = (int32_t)sch.tiles.size() - it.tile_begin;
+            it.partial_slot = -1;
+            sch.items.push_back(it);
+        }
+    }
+
+    // ---- work order: longest lists first (the block scheduler hands items out in this order, so
+    // the short border patches fill the tail); stable, so equal items keep their raster order
+    std::stable_sort(sch.items.begin(), sch.items.end(),
+                     [](const clear_work_item_t &a, const clear_work_item_t &b) { return a.tile_count > b.tile_count; });
+
+    sch.max_item_tiles = 0;
+    sch.executed_pairs = 0;
+    for (const auto &it : sch.items) {
+        sch.max_item_tiles = std::max(sch.max_item_tiles, it.tile_count);
+        sch.executed_pairs += (int64_t)it.tile_count * kTileTokens * kTileTokens;
+    }
+}
+
+}  // namespace clear

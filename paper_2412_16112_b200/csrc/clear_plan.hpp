@@ -1,0 +1,50 @@
+// Host-side schedule of the CLEAR attention kernels (no CUDA in this header).
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "clear_attn.h"
+
+namespace clear {
+
+constexpr int kTileH = 8;      // query / key patch: 8 grid rows ...
+constexpr int kTileW = 16;     // ... by 16 grid columns = 128 tokens
+constexpr int kTileTokens = 128;
+constexpr int kSplitTargetTiles = 64;  // key tiles per split of a text-query tile
+
+struct Shape {
+    int B = 0, H = 0, grid_h = 0, grid_w = 0, n_text = 0, head_dim = 0;
+    float radius = 0.f;
+    int dtype = 0;
+    int kernel = 0;
+    bool operator==(const Shape &o) const
+    {
+        return B == o.B && H == o.H && grid_h == o.grid_h && grid_w == o.grid_w && n_text == o.n_text &&
+               head_dim == o.head_dim && radius == o.radius && dtype == o.dtype && kernel == o.kernel;
+    }
+};
+
+struct Schedule {
+    int64_t thr = 0;                     // ceil(radius^2): allowed iff dx^2 + dy^2 < thr (Eq. 3)
+    std::vector<int32_t> half_width;     // half_width[dy] = max |dx| allowed at row offset dy
+    std::vector<clear_work_item_t> items;
+    std::vector<clear_kv_tile_t> tiles;
+    int n_text_tiles = 0;                // text-query tiles of 128 rows
+    int n_text_splits = 0;               // splits per text-query tile (1 = no partial results)
+    int n_partial_slots = 0;
+    int max_item_tiles = 0;
+    int64_t sum_mask = 0;
+    int64_t executed_pairs = 0;
+};
+
+// Validate the arguments every entry point shares.  Returns a clear_status.
+int validate_shape(const Shape &s);
+
+// Integer geometry common to both kernels: thr, half_width[], sum_mask.
+void build_geometry(const Shape &s, Schedule &sch);
+
+// Work items and key-tile lists of the tensor-core kernel (calls build_geometry first).
+void build_tile_schedule(const Shape &s, Schedule &sch);
+
+}  // namespace clear

@@ -1,0 +1,322 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle, element by element
+on small cases and on sampled rows at the full workload sizes."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import clear_oracle as oracle
+from paper_2412_16112_b200 import binding as clear
+from paper_2412_16112_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+# tolerances: bf16 inputs / fp32 accumulation, and the fp32 path
+BF16_MAX, BF16_MEAN = 2e-2, 2e-3
+F32_MAX = 1e-5
+
+
+def dev():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    return torch.device("cuda:0")
+
+
+def run_plan(q, k, v, gh, gw, T, r, scale, kernel, dtype=clear.BF16):
+    B, H, N, d = q.shape
+    plan = clear.Plan(B, H, gh, gw, T, d, r, dtype=dtype, kernel=kernel)
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    out = torch.full_like(qd, float("nan"))
+    plan.forward(qd, kd, vd, out, scale)
+    plan.check()
+    res = out.cpu()
+    plan.destroy()
+    return res
+
+
+def assert_close_bf16(got, want, what=""):
+    err = np.abs(got.double().numpy() - want)
+    assert np.isfinite(err).all(), f"{what}: non-finite output"
+    rel = np.linalg.norm(err) / max(np.linalg.norm(want), 1e-30)
+    assert err.max() <= BF16_MAX and err.mean() <= BF16_MEAN, \
+        f"{what}: max {err.max():.3e} mean {err.mean():.3e} rel {rel:.3e}"
+    return err.max(), err.mean(), rel
+
+
+def sample_rows(w, heads, n_random, rng):
+    """(b, h, i) triples: text rows, grid corners / edges / tile seams, random image rows."""
+    gh, gw, T = w.grid_h, w.grid_w, w.n_text
+    ys = sorted({0, 1, 7, 8, 9, gh // 2 - 1, gh // 2, gh - 9, gh - 8, gh - 2, gh - 1} & set(range(gh)))
+    xs = sorted({0, 1, 15, 16, 17, gw // 2 - 1, gw // 2, gw - 17, gw - 16, gw - 2, gw - 1} & set(range(gw)))
+    rows = []
+    for h in heads:
+        text = sorted({0, 1, 127, 128, T // 2, T - 1} & set(range(T)))
+        rows += [(0, h, i) for i in text]
+        rows += [(0, h, T + y * gw + x) for y in ys for x in xs]
+        rows += [(0, h, T + int(p)) for p in rng.integers(0, gh * gw, n_random)]
+    return np.array(rows, dtype=np.int64)
+
+
+# ----------------------------------------------------------------------------------------------
+# fp32 path (config 0) and the CUDA-core kernel
+# ----------------------------------------------------------------------------------------------
+def test_c0_tiny_fp32_matches_oracle_everywhere():
+    w = workloads.WORKLOADS["c0_tiny_f32"]
+    q, k, v = workloads.make_inputs(w)
+    want = oracle.attn(q, k, v, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale)
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    out = torch.full_like(qd, float("nan"))
+    clear.clear_attn_fwd_f32(qd, kd, vd, out, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale)
+    torch.cuda.synchronize()
+    err = np.abs(out.cpu().double().numpy() - want)
+    assert err.max() <= F32_MAX, err.max()
+
+
+@pytest.mark.parametrize("gh,gw,T,r,d,dtype", [
+    (13, 19, 7, 4.0, 64, "f32"), (9, 5, 0, 2.5, 40, "f32"), (6, 33, 130, 1.0, 128, "f32"),
+    (12, 12, 3, 100.0, 256, "f32"), (13, 19, 7, 4.0, 64, "bf16"), (10, 21, 33, 3.0, 96, "bf16"),
+    (16, 16, 16, 4.0, 128, "bf16"),
+])
+def test_simt_kernel_small_shapes(gh, gw, T, r, d, dtype):
+    q, k, v = workloads.make_custom(2, 2, gh, gw, T, d, dtype=dtype, qk_norm=(dtype == "bf16"), seed=gh * 100 + gw)
+    scale = 1 / math.sqrt(d)
+    want = oracle.attn(q, k, v, gh, gw, T, r, scale)
+    code = clear.BF16 if dtype == "bf16" else clear.F32
+    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_SIMT, dtype=code)
+    if dtype == "f32":
+        assert np.abs(got.double().numpy() - want).max() <= F32_MAX
+    else:
+        assert_close_bf16(got, want, "simt bf16")
+
+
+def test_simt_kernel_takes_a_negative_scale():
+    gh, gw, T, d = 8, 9, 4, 64
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, dtype="f32", qk_norm=False, seed=5)
+    want = oracle.attn(q, k, v, gh, gw, T, 3.0, -0.2)
+    got = run_plan(q, k, v, gh, gw, T, 3.0, -0.2, clear.KERNEL_SIMT, dtype=clear.F32)
+    assert np.abs(got.double().numpy() - want).max() <= F32_MAX
+
+
+# ----------------------------------------------------------------------------------------------
+# tensor-core kernel, small shapes: every element
+# ----------------------------------------------------------------------------------------------
+TC_SMALL = [
+    # gh, gw, T, r, d
+    (16, 16, 16, 4.0, 64),       # config 0's shape through the bf16 kernel
+    (16, 16, 16, 4.0, 128),
+    (8, 16, 0, 1.0, 128),        # one patch, no text, self only
+    (13, 19, 7, 4.0, 128),       # ragged patches on both axes, ragged text tile
+    (24, 40, 130, 8.0, 128),     # text tail of 2 tokens in a second tile
+    (9, 33, 0, 5.5, 64),         # no text, non-integer radius
+    (40, 24, 256, 16.0, 128),
+    (20, 50, 3, 100.0, 128),     # radius beyond the diagonal: full attention
+    (1, 70, 2, 3.0, 64),         # single-row grid
+    (33, 1, 0, 2.5, 128),        # single-column grid
+    (32, 48, 128, 2.0, 128),
+]
+
+
+@pytest.mark.parametrize("gh,gw,T,r,d", TC_SMALL)
+def test_tc_kernel_small_shapes(gh, gw, T, r, d):
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=gh * 1000 + gw * 10 + T)
+    scale = 1 / math.sqrt(d)
+    want = oracle.attn(q, k, v, gh, gw, T, r, scale)
+    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05)
+    assert_close_bf16(got, want, f"tc {gh}x{gw}+{T} r={r} d={d}")
+
+
+def test_tc_kernel_split_text_rows_small():
+    """N large enough that the text-query rows are split over key ranges and merged."""
+    gh, gw, T, r, d = 96, 96, 200, 6.0, 128
+    plan = clear.Plan(1, 1, gh, gw, T, d, r, host_only=True)
+    assert plan.info().n_text_splits > 1
+    q, k, v = workloads.make_custom(1, 1, gh, gw, T, d, seed=77)
+    scale = 1 / math.sqrt(d)
+    rng = np.random.default_rng(0)
+    rows = np.array([(0, 0, i) for i in list(range(0, T, 7)) + [T - 1] +
+                     [T + int(p) for p in rng.integers(0, gh * gw, 200)]], dtype=np.int64)
+    want = oracle.attn_rows(q, k, v, gh, gw, T, r, scale, rows)
+    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05)
+    assert_close_bf16(got[rows[:, 0], rows[:, 1], rows[:, 2]], want, "split text rows")
+
+
+def test_tc_kernel_large_logits_exercise_the_rescale_path():
+    """Un-normalised Q, K: row maxima jump by far more than the lazy-rescale threshold."""
+    gh, gw, T, r, d = 24, 32, 64, 6.0, 128
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, qk_norm=False, seed=9)
+    scale = 1.0
+    want = oracle.attn(q, k, v, gh, gw, T, r, scale)
+    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05)
+    assert_close_bf16(got, want, "large logits")
+
+
+# ----------------------------------------------------------------------------------------------
+# mask exactness through bf16: uniform softmax reads membership and counts
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("kernel", [clear.KERNEL_TCGEN05, clear.KERNEL_SIMT])
+@pytest.mark.parametrize("gh,gw,T,r", [(24, 40, 5, 8.0), (19, 23, 0, 4.0), (16, 48, 130, 3.0)])
+def test_zero_queries_read_back_the_mask(kernel, gh, gw, T, r):
+    """Q = 0: out_i = mean of V over the allowed set.  V column c is one-hot on a planted key, so
+    out is 1/|A_i| where the key is allowed and exactly 0 elsewhere; a constant column reads 1."""
+    d = 64
+    N = T + gh * gw
+    rng = np.random.default_rng(3)
+    planted = rng.choice(np.arange(T, N), size=d - 2, replace=False)
+    if T > 0:
+        planted[0] = 0                                   # one text key
+    v = torch.zeros(1, 1, N, d)
+    for c, j in enumerate(planted):
+        v[0, 0, j, c] = 1.0
+    v[..., d - 1] = 1.0
+    q = torch.zeros(1, 1, N, d)
+    k = torch.randn(1, 1, N, d, generator=torch.Generator().manual_seed(1))
+    q, k, v = (t.to(torch.bfloat16) for t in (q, k, v))
+    got = run_plan(q, k, v, gh, gw, T, r, 1.0, kernel).double().numpy()[0, 0]
+    _, counts = oracle.mask_counts(gh, gw, T, r)
+    for i in range(N):
+        row = oracle.mask_row(i, gh, gw, T, r)
+        member = row[planted].astype(bool)
+        assert np.all(got[i, :d - 2][~member] == 0.0), f"query {i} sees a key outside its window"
+        np.testing.assert_allclose(got[i, :d - 2][member], 1.0 / counts[i], rtol=1.5e-2)
+        assert abs(got[i, d - 1] - 1.0) < 1e-2
+
+
+def test_planted_key_at_the_radius_threshold():
+    """A key with a dominant logit at squared distance thr-1 takes over the output; at thr it must not."""
+    gh, gw, T, r, d = 24, 40, 4, 5.0, 128           # thr = 25: (3, 4) is at d2 = 25, (0, 4) at 16, (2, 4) at 20
+    N = T + gh * gw
+    g = torch.Generator().manual_seed(2)
+    q = torch.randn(1, 1, N, d, generator=g) * 0.05
+    k = torch.randn(1, 1, N, d, generator=g) * 0.05
+    v = torch.randn(1, 1, N, d, generator=g)
+    qy, qx = 11, 17                                  # not aligned with the patch lattice
+    qi = T + qy * gw + qx
+    q[0, 0, qi] = 0.0
+    q[0, 0, qi, 0] = 8.0
+    inside = T + (qy + 2) * gw + (qx + 4)            # d2 = 20 < 25
+    outside = T + (qy + 3) * gw + (qx + 4)           # d2 = 25: excluded by the strict inequality
+    wrap = T + (qy + 1) * gw + (qx + 4 - gw)         # next row, far left: token-adjacent only
+    for j, val in ((inside, 4.0), (outside, 8.0), (wrap, 8.0)):
+        k[0, 0, j] = 0.0
+        k[0, 0, j, 0] = val
+    q, k, v = (t.to(torch.bfloat16) for t in (q, k, v))
+    want = oracle.attn_rows(q, k, v, gh, gw, T, r, 1.0, [[0, 0, qi]])[0]
+    assert np.abs(want - v[0, 0, inside].double().numpy()).max() < 1e-2   # the oracle picks `inside`
+    for kernel in (clear.KERNEL_TCGEN05, clear.KERNEL_SIMT):
+        got = run_plan(q, k, v, gh, gw, T, r, 1.0, kernel)[0, 0, qi].double().numpy()
+        assert np.abs(got - want).max() < 2e-2
+
+
+# ----------------------------------------------------------------------------------------------
+# full workload sizes: sampled rows against the oracle, whole-output properties
+# ----------------------------------------------------------------------------------------------
+_INPUT_CACHE = {}
+
+
+def full_inputs(w):
+    key = (w.seed, w.grid_h, w.grid_w)
+    if key not in _INPUT_CACHE:
+        _INPUT_CACHE.clear()
+        _INPUT_CACHE[key] = workloads.make_inputs(w)
+    return _INPUT_CACHE[key]
+
+
+@pytest.mark.parametrize("name", ["c1_1024px_r8", "c2_2048px_r16", "c3_4096px_r8", "c3_4096px_r16",
+                                  "c3_4096px_r32", "c3_192x320_r16", "c4_8k_r16"])
+def test_full_size_workloads_on_sampled_rows(name):
+    w = workloads.WORKLOADS[name]
+    q, k, v = full_inputs(w)
+    rng = np.random.default_rng(w.seed)
+    rows = sample_rows(w, heads=[0, w.H // 2, w.H - 1], n_random=64, rng=rng)
+    want = oracle.attn_rows(q, k, v, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale, rows)
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    out = torch.full_like(qd, float("nan"))
+    # the launch configuration the benchmark times: the cached-plan entry point on the current stream
+    clear.clear_attn_fwd(qd, kd, vd, out, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all(), "some output element was never written"
+    got = out[rows[:, 0], rows[:, 1], rows[:, 2]].cpu()
+    assert_close_bf16(got, want, name)
+    # any-size property: every output is a convex combination of V rows
+    vmax = vd.float().amax(dim=2, keepdim=True)
+    vmin = vd.float().amin(dim=2, keepdim=True)
+    o = out.float()
+    assert bool(((o <= vmax + 2e-2) & (o >= vmin - 2e-2)).all())
+    del qd, kd, vd, out
+    clear.clear_cache_clear()
+    torch.cuda.empty_cache()
+
+
+def test_rows_stay_normalised_at_full_size():
+    """V = 1 everywhere -> out = 1 everywhere (checks the row sums of every tile of the 2048px config)."""
+    w = workloads.WORKLOADS["c2_2048px_r16"]
+    q, k, _ = full_inputs(w)
+    qd, kd = q.to(dev()), k.to(dev())
+    vd = torch.ones_like(qd)
+    out = torch.full_like(qd, float("nan"))
+    clear.clear_attn_fwd(qd, kd, vd, out, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale)
+    torch.cuda.synchronize()
+    assert float((out.float() - 1.0).abs().max()) < 1e-2
+    clear.clear_cache_clear()
+
+
+# ----------------------------------------------------------------------------------------------
+# robustness of the boundary
+# ----------------------------------------------------------------------------------------------
+def test_guard_bands_repeat_calls_and_streams():
+    gh, gw, T, r, d = 24, 40, 130, 8.0, 128
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=21)
+    scale = 1 / math.sqrt(d)
+    n = q.numel()
+    guard = 4096
+    buf = torch.full((n + 2 * guard,), -7.0, dtype=torch.bfloat16, device=dev())
+    out = buf[guard: guard + n].view(q.shape)
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    plan = clear.Plan(1, 2, gh, gw, T, d, r, kernel=clear.KERNEL_TCGEN05)
+    plan.forward(qd, kd, vd, out, scale)
+    plan.check()
+    first = out.clone()
+    assert bool((buf[:guard] == -7.0).all()) and bool((buf[guard + n:] == -7.0).all())
+    # same plan again, on a side stream
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    out.fill_(float("nan"))
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        plan.forward(qd, kd, vd, out, scale, stream=side)
+    side.synchronize()
+    plan.check()
+    assert torch.equal(out, first), "the kernel is not deterministic across calls"
+    # other output buffer: the plan's cached tensor maps must follow the pointers
+    out2 = torch.full_like(qd, float("nan"))
+    plan.forward(qd, kd, vd, out2, scale)
+    plan.check()
+    assert torch.equal(out2, first)
+    want = oracle.attn(q, k, v, gh, gw, T, r, scale)
+    assert_close_bf16(first.cpu(), want, "guarded call")
+    plan.destroy()
+
+
+def test_device_side_argument_errors():
+    lib = clear.load()
+    x = torch.zeros(1, 1, 16 * 16 + 16, 64, dtype=torch.bfloat16, device=dev())
+    p = x.data_ptr()
+    assert lib.clear_attn_fwd(p, p, p, p + 2, 1, 1, 16, 16, 16, 64, 4.0, 0.125, None) == clear.ERR_MISALIGNED
+    assert lib.clear_attn_fwd(p, p, p, None, 1, 1, 16, 16, 16, 64, 4.0, 0.125, None) == clear.ERR_INVALID_ARG
+    plan = clear.Plan(1, 1, 16, 16, 16, 64, 4.0, kernel=clear.KERNEL_TCGEN05)
+    out = torch.empty_like(x)
+    assert lib.clear_attn_fwd_planned(plan.handle, p, p, p, out.data_ptr(), -1.0, None) == clear.ERR_UNSUPPORTED
+    plan.destroy()
+
+
+def test_host_tensor_entry_point():
+    gh, gw, T, r, d = 16, 32, 20, 4.0, 128
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=31)
+    scale = 1 / math.sqrt(d)
+    plan = clear.Plan(1, 2, gh, gw, T, d, r)
+    qh, kh, vh = (t.pin_memory() for t in (q, k, v))
+    oh = torch.empty_like(q).pin_memory()
+    plan.forward_host(qh, kh, vh, oh, scale)
+    want = oracle.attn(q, k, v, gh, gw, T, r, scale)
+    assert_close_bf16(oh, want, "host entry point")
+    plan.destroy()
