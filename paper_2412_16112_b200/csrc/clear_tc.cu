@@ -271,7 +271,8 @@ clear_tc_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 }
             }
 
-            if (!wait_bar(b_s, ph, abort_flag, prm.status, 7)) { alive = false; break; }
+            // warp-uniform outcome: the tcgen05.ld / st below need the whole warp
+            if (!__all_sync(0xffffffffu, wait_bar(b_s, ph, abort_flag, prm.status, 7))) { alive = false; break; }
             ptx::tc_fence_after();
             uint32_t s[4][32];
 #pragma unroll
@@ -354,7 +355,7 @@ clear_tc_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         }
 
         // ---- epilogue: wait for the last PV, then normalise and store ---------------------------------
-        if (alive) alive = wait_bar(b_o, (uint32_t)((n_tiles - 1) & 1), abort_flag, prm.status, 8);
+        if (alive) alive = __all_sync(0xffffffffu, wait_bar(b_o, (uint32_t)((n_tiles - 1) & 1), abort_flag, prm.status, 8));
         if (alive) {
             ptx::tc_fence_after();
             if (item.partial_slot >= 0) {

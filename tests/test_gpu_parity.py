@@ -182,28 +182,33 @@ def test_zero_queries_read_back_the_mask(kernel, gh, gw, T, r):
 
 
 def test_planted_key_at_the_radius_threshold():
-    """A key with a dominant logit at squared distance thr-1 takes over the output; at thr it must not."""
-    gh, gw, T, r, d = 24, 40, 4, 5.0, 128           # thr = 25: (3, 4) is at d2 = 25, (0, 4) at 16, (2, 4) at 20
+    """A key with a dominant logit at squared distance thr-5 takes over the output; a stronger one at
+    exactly thr must not, nor one that is next in token order but a grid-width away."""
+    gh, gw, T, r, d = 24, 40, 4, 5.0, 128           # thr = 25: offset (3, 4) is at d2 = 25, (2, 4) at 20
     N = T + gh * gw
     g = torch.Generator().manual_seed(2)
     q = torch.randn(1, 1, N, d, generator=g) * 0.05
     k = torch.randn(1, 1, N, d, generator=g) * 0.05
     v = torch.randn(1, 1, N, d, generator=g)
     qy, qx = 11, 17                                  # not aligned with the patch lattice
-    qi = T + qy * gw + qx
-    q[0, 0, qi] = 0.0
-    q[0, 0, qi, 0] = 8.0
+    qa = T + qy * gw + qx
+    qb = T + 5 * gw + (gw - 1)                       # last column of row 5
+    for qi in (qa, qb):
+        q[0, 0, qi] = 0.0
+        q[0, 0, qi, 0] = 8.0
     inside = T + (qy + 2) * gw + (qx + 4)            # d2 = 20 < 25
     outside = T + (qy + 3) * gw + (qx + 4)           # d2 = 25: excluded by the strict inequality
-    wrap = T + (qy + 1) * gw + (qx + 4 - gw)         # next row, far left: token-adjacent only
+    wrap = T + 6 * gw + 0                            # the token right after qb, 39 columns away
     for j, val in ((inside, 4.0), (outside, 8.0), (wrap, 8.0)):
         k[0, 0, j] = 0.0
         k[0, 0, j, 0] = val
     q, k, v = (t.to(torch.bfloat16) for t in (q, k, v))
-    want = oracle.attn_rows(q, k, v, gh, gw, T, r, 1.0, [[0, 0, qi]])[0]
-    assert np.abs(want - v[0, 0, inside].double().numpy()).max() < 1e-2   # the oracle picks `inside`
+    rows = [[0, 0, qa], [0, 0, qb]]
+    want = oracle.attn_rows(q, k, v, gh, gw, T, r, 1.0, rows)
+    assert np.abs(want[0] - v[0, 0, inside].double().numpy()).max() < 1e-2   # the oracle picks `inside`
+    assert np.abs(want[1] - v[0, 0, wrap].double().numpy()).max() > 0.5      # and never sees `wrap`
     for kernel in (clear.KERNEL_TCGEN05, clear.KERNEL_SIMT):
-        got = run_plan(q, k, v, gh, gw, T, r, 1.0, kernel)[0, 0, qi].double().numpy()
+        got = run_plan(q, k, v, gh, gw, T, r, 1.0, kernel)[0, 0, [qa, qb]].double().numpy()
         assert np.abs(got - want).max() < 2e-2
 
 
