@@ -39,7 +39,8 @@ typedef enum clear_status {
     CLEAR_ERR_PLAN_MISMATCH = -4,  /* plan used on another device / with a kernel it was not built for */
     CLEAR_ERR_CUDA = -5,           /* a CUDA runtime or driver call failed (see clear_last_cuda_error) */
     CLEAR_ERR_DEVICE_TIMEOUT = -6, /* a bounded wait inside a kernel expired; outputs are invalid    */
-    CLEAR_ERR_NO_MEMORY = -7       /* host or device allocation failed                               */
+    CLEAR_ERR_NO_MEMORY = -7,      /* host or device allocation failed                               */
+    CLEAR_ERR_TOO_LARGE = -8       /* shape exceeds a fixed capacity of clear_attn_fwd_static        */
 } clear_status;
 
 typedef enum clear_dtype { CLEAR_BF16 = 0, CLEAR_F32 = 1 } clear_dtype;
@@ -144,6 +145,37 @@ int clear_attn_fwd_planned(const clear_plan_t *plan, const void *q, const void *
  * and DEVICE_TIMEOUT. */
 int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_host,
                         const void *v_host, void *out_host, float scale, void *stream);
+
+/* Fixed capacities of clear_attn_fwd_static (one static device array of about 33.3 MiB in total). */
+#define CLEAR_STATIC_SCRATCH_BYTES (32u << 20) /* split-KV partial results of the text-query rows      */
+#define CLEAR_STATIC_MAX_ITEMS 8192            /* work items per (batch, head)                          */
+#define CLEAR_STATIC_MAX_TILES 65536           /* key-tile list entries per (batch, head)               */
+#define CLEAR_STATIC_MAX_HALF_WIDTH 1024       /* rows an image query can reach upwards, plus one       */
+
+/* bf16 forward pass on the tensor-core kernel that never allocates device memory.  (The paper has no
+ * counterpart: this is an interface variant, not a step of the method.)
+ *
+ * Who needs it: code that may not call cudaMalloc at the point where attention runs -- a host running
+ * under a fixed, pre-partitioned memory budget, a plug-in whose embedding framework owns every device
+ * byte, or a process that has already handed all free memory to a caching allocator, where a driver
+ * allocation would fail or stall the other streams.  The planned entry points allocate schedule tables
+ * and a split-KV workspace per plan; this one keeps them in one file-scope device array inside the
+ * library image, so every GPU that loads the library holds those ~33.3 MiB until the process exits.
+ *
+ * Same tensors, layout and mathematics as clear_attn_fwd (results are identical bit for bit); head_dim
+ * must be 64 or 128 and scale > 0.  It calls no cudaMalloc / cudaFree and no allocating library routine;
+ * it does enqueue small table copies and one 4-byte memset on `stream`.
+ * - The first call on a device looks up the array's device address (set-up); make that call with the
+ *   device current and before starting any stream capture.
+ * - Shapes whose tables or partial results exceed the CLEAR_STATIC_* capacities are rejected with
+ *   CLEAR_ERR_TOO_LARGE (the 2048px FLUX shape fits; the 4096px and 8K shapes do not).
+ * - All calls on a device share the array, which keeps the last call's contents; the call re-uploads the
+ *   tables when the shape changes and clears the status word every time.  Two calls that overlap on the
+ *   GPU (different streams without ordering) race on it: order them.
+ * - Device-side wait expiries are not reported by this entry point.
+ * Errors: INVALID_ARG, UNSUPPORTED, MISALIGNED, TOO_LARGE, NO_MEMORY (host), CUDA. */
+int clear_attn_fwd_static(const void *q, const void *k, const void *v, void *out, int B, int H, int grid_h,
+                          int grid_w, int n_text, int head_dim, float radius, float scale, void *stream);
 
 /* Fill `info` from the plan (host only, no CUDA call).  Errors: INVALID_ARG. */
 int clear_plan_info(const clear_plan_t *plan, clear_plan_info_t *info);

@@ -15,7 +15,7 @@ from . import build as _build
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_PLAN_MISMATCH = -1, -2, -3, -4
-ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY = -5, -6, -7
+ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY, ERR_TOO_LARGE = -5, -6, -7, -8
 BF16, F32 = 0, 1
 KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05 = 0, 1, 2
 TILE_LINEAR, TILE_MASKED = 1, 2
@@ -24,7 +24,7 @@ EXPORTS = [
     "clear_attn_fwd", "clear_attn_fwd_f32", "clear_plan_create", "clear_plan_create_host",
     "clear_plan_tables", "clear_attn_fwd_planned", "clear_attn_fwd_host", "clear_plan_info",
     "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
-    "clear_last_cuda_error",
+    "clear_last_cuda_error", "clear_attn_fwd_static",
 ]
 
 
@@ -74,6 +74,7 @@ def load() -> ctypes.CDLL:
         fwd_args = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp]
         lib.clear_attn_fwd.argtypes = fwd_args
         lib.clear_attn_fwd_f32.argtypes = fwd_args
+        lib.clear_attn_fwd_static.argtypes = fwd_args
         plan_args = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, f32, i32, i32]
         lib.clear_plan_create.argtypes = plan_args
         lib.clear_plan_create_host.argtypes = plan_args
@@ -147,6 +148,19 @@ def clear_attn_fwd_f32(q, k, v, out, grid_h, grid_w, n_text, radius, scale, stre
     B, H, _, d = q.shape
     _check(load().clear_attn_fwd_f32(*ptrs, B, H, grid_h, grid_w, n_text, d, float(radius), float(scale),
                                      _stream_ptr(stream)), "clear_attn_fwd_f32")
+    return out
+
+
+def clear_attn_fwd_static(q, k, v, out, grid_h, grid_w, n_text, radius, scale, stream=None):
+    """bf16 forward pass that allocates no device memory: its tables and split-KV scratch live in a
+    fixed-size array inside the library.  Meant for callers that cannot call cudaMalloc where attention
+    runs (fixed memory budgets, plug-ins, processes whose caching allocator already owns the device).
+    Shapes beyond the fixed capacities raise ``ClearError`` with status ``ERR_TOO_LARGE``; calls on one
+    device share the array, so do not let two of them overlap on the GPU."""
+    ptrs = _tensor_args(q, k, v, out, BF16)
+    B, H, _, d = q.shape
+    _check(load().clear_attn_fwd_static(*ptrs, B, H, grid_h, grid_w, n_text, d, float(radius), float(scale),
+                                        _stream_ptr(stream)), "clear_attn_fwd_static")
     return out
 
 

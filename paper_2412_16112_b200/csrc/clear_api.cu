@@ -358,6 +358,7 @@ const char *clear_status_string(int status)
         case CLEAR_ERR_CUDA: return "CUDA call failed";
         case CLEAR_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
         case CLEAR_ERR_NO_MEMORY: return "out of memory";
+        case CLEAR_ERR_TOO_LARGE: return "shape exceeds a fixed capacity of the no-allocation entry point";
         default: return "unknown status";
     }
 }
