@@ -191,7 +191,7 @@ def run_ours(args, w):
     stream = torch.cuda.current_stream()
     small = 4 * qd.numel() * qd.element_size() <= 2 * 126e6
     flush = torch.empty(int(256e6), dtype=torch.uint8, device=dev) if small else None
-    launches_per_call = 1 + (1 if (info.kernel == clear.KERNEL_TCGEN05 and info.n_text_splits > 1) else 0)
+    launches_per_call = 1 + (1 if (info.kernel != clear.KERNEL_SIMT and info.n_text_splits > 1) else 0)
 
     def barrier():
         if dist is not None:
@@ -265,13 +265,14 @@ def run_ours(args, w):
                 traffic = json.load(f).get(w.name)
         except Exception:
             traffic = None
-    if info.kernel == clear.KERNEL_TCGEN05:
+    if info.kernel != clear.KERNEL_SIMT:
         roofline = {"bound": "tensor", "achieved": per_gpu_tflops, "peak": peak, "unit": "TFLOP/s",
                     "frac": per_gpu_tflops / peak, "traffic": traffic, "peak_kind": f"{peaks_kind} bf16 burst",
                     "frac_of_sustained": per_gpu_tflops / float(peaks.get("bf16_tflops_sustained", peak)),
                     "executed_tflops": per_gpu_tflops * info.executed_pairs / info.sum_mask,
                     "geometric_efficiency": info.sum_mask / info.executed_pairs,
-                    "kernel": "clear_tc_kernel (+ combine kernel inside the same events)"}
+                    "kernel": ("clear_ws_kernel" if info.kernel == clear.KERNEL_TCGEN05_WS else "clear_tc_kernel") +
+                              " (+ combine kernel inside the same events)"}
     else:
         # fp32 CUDA-core kernel: 128 FMA lanes x 2 flops per SM per clock
         alu_peak = 148 * 128 * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12

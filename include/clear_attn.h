@@ -46,10 +46,19 @@ typedef enum clear_status {
 typedef enum clear_dtype { CLEAR_BF16 = 0, CLEAR_F32 = 1 } clear_dtype;
 
 /* Which kernel a plan drives.
- *   AUTO    : TCGEN05 when it applies (bf16, head_dim 64 or 128, scale > 0 at call time), else SIMT.
- *   SIMT    : exact-order fp32 CUDA-core kernel; any head_dim <= 256, bf16 or fp32 tensors.
- *   TCGEN05 : block-sparse flash-style kernel on the 5th-generation tensor cores (TMA + TMEM). */
-typedef enum clear_kernel { CLEAR_KERNEL_AUTO = 0, CLEAR_KERNEL_SIMT = 1, CLEAR_KERNEL_TCGEN05 = 2 } clear_kernel;
+ *   AUTO       : TCGEN05_WS when it applies (bf16, head_dim 64 or 128, scale > 0 at call time), else SIMT.
+ *   SIMT       : exact-order fp32 CUDA-core kernel; any head_dim <= 256, bf16 or fp32 tensors.
+ *   TCGEN05    : block-sparse flash-style kernel on the 5th-generation tensor cores (TMA + TMEM), one
+ *                128-query tile per thread block, two blocks per SM.
+ *   TCGEN05_WS : the same mathematics as a persistent, warp-specialised kernel: one block per SM walks a
+ *                work queue; each work item is a PAIR of 128-query tiles (two vertically adjacent grid
+ *                patches, or two text tiles) that share every key/value tile both of them need. */
+typedef enum clear_kernel {
+    CLEAR_KERNEL_AUTO = 0,
+    CLEAR_KERNEL_SIMT = 1,
+    CLEAR_KERNEL_TCGEN05 = 2,
+    CLEAR_KERNEL_TCGEN05_WS = 3
+} clear_kernel;
 
 typedef struct clear_plan clear_plan_t; /* opaque */
 
@@ -94,6 +103,42 @@ typedef struct clear_work_item {
     int32_t reserved;
 } clear_work_item_t;
 
+/* ---- schedule tables of the TCGEN05_WS kernel ------------------------------------------------ */
+
+enum {
+    CLEAR_STEP_USE0 = 1,    /* query tile 0 of the pair visits its key tile in this step             */
+    CLEAR_STEP_USE1 = 2,    /* query tile 1 of the pair visits its key tile in this step             */
+    CLEAR_STEP_SHARED = 4,  /* both visit the SAME key tile (x0, y0): it is staged once             */
+    CLEAR_STEP_LINEAR = 8,  /* key tiles of this step are 128 consecutive tokens, else 2-D patches  */
+    CLEAR_STEP_MASKED0 = 16, /* tile 0 must apply Eq. 3 / n_valid0 to its key tile                  */
+    CLEAR_STEP_MASKED1 = 32  /* tile 1 likewise                                                     */
+};
+
+/* One step of a pair item: each query tile of the pair multiplies against one key tile. */
+typedef struct clear_pair_step {
+    int32_t x0, y0;     /* key tile of query tile 0 (and of tile 1 when SHARED); as clear_kv_tile_t */
+    int32_t x1, y1;     /* key tile of query tile 1 when not SHARED                                 */
+    int32_t flags;      /* CLEAR_STEP_* bits                                                        */
+    int32_t n_valid0;   /* linear tiles: keys [0, n_valid) of the tile exist / are allowed          */
+    int32_t n_valid1;
+    int32_t load_base;  /* key/value tiles the item has staged before this step (K and V counted
+                           separately): position of this step's first stage in the block's ring     */
+} clear_pair_step_t;
+
+/* One unit of work of the TCGEN05_WS kernel: two 128-query tiles walking one step list. */
+typedef struct clear_pair_item {
+    int32_t kind;          /* 0 = two vertically adjacent 8 x 16 image patches, 1 = two text tiles   */
+    int32_t n_sides;       /* 2, or 1 when the second tile does not exist                            */
+    int32_t qx;            /* image: grid column of both patches; text: first token of tile 0        */
+    int32_t qy0, qy1;      /* image: grid row of patch 0 / patch 1; text: unused (tile 1 = qx + 128) */
+    int32_t n_rows0, n_rows1; /* queries of each tile that exist                                     */
+    int32_t step_begin;    /* first entry of its list in the step table                              */
+    int32_t step_count;    /* length of the list (>= 1)                                              */
+    int32_t n_loads;       /* key and value tiles its steps stage in total                           */
+    int32_t partial_slot0; /* -1: tile 0 writes final outputs; else its split-KV partial-result slot */
+    int32_t partial_slot1;
+} clear_pair_item_t;
+
 /* Eq. 1 under the mask of Eq. 3 for bf16 tensors, fp32 accumulation, bf16 output.
  * A plan for the shape is looked up in (or added to) a process-wide cache, so the first call for
  * a shape allocates and copies small tables; later calls only launch kernels.
@@ -130,6 +175,11 @@ int clear_plan_create_host(clear_plan_t **plan, int B, int H, int grid_h, int gr
 int clear_plan_tables(const clear_plan_t *plan, const clear_work_item_t **items, int32_t *n_items,
                       const clear_kv_tile_t **tiles, int32_t *n_tiles, const int32_t **half_width,
                       int32_t *n_half_width);
+
+/* The same for a TCGEN05_WS plan: its pair items (text items first, then image items, longest step
+ * lists first) and their steps.  Empty for other plans.  Errors: INVALID_ARG. */
+int clear_plan_pair_tables(const clear_plan_t *plan, const clear_pair_item_t **items, int32_t *n_items,
+                           const clear_pair_step_t **steps, int32_t *n_steps);
 
 /* Forward pass with an explicit plan.  Tensor dtype is the plan's.  Calls on one plan share its
  * workspace: run them on one stream, or order them yourself.

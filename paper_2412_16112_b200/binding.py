@@ -17,14 +17,15 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_PLAN_MISMATCH = -1, -2, -3, -4
 ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY, ERR_TOO_LARGE = -5, -6, -7, -8
 BF16, F32 = 0, 1
-KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05 = 0, 1, 2
+KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_TCGEN05_WS = 0, 1, 2, 3
 TILE_LINEAR, TILE_MASKED = 1, 2
+STEP_USE0, STEP_USE1, STEP_SHARED, STEP_LINEAR, STEP_MASKED0, STEP_MASKED1 = 1, 2, 4, 8, 16, 32
 
 EXPORTS = [
     "clear_attn_fwd", "clear_attn_fwd_f32", "clear_plan_create", "clear_plan_create_host",
     "clear_plan_tables", "clear_attn_fwd_planned", "clear_attn_fwd_host", "clear_plan_info",
     "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
-    "clear_last_cuda_error", "clear_attn_fwd_static",
+    "clear_last_cuda_error", "clear_attn_fwd_static", "clear_plan_pair_tables",
 ]
 
 
@@ -50,6 +51,17 @@ class KvTile(ctypes.Structure):
 class WorkItem(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("kind", "qx", "qy", "n_rows", "tile_begin", "tile_count", "partial_slot", "reserved")]
+
+
+class PairStep(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("x0", "y0", "x1", "y1", "flags", "n_valid0", "n_valid1", "load_base")]
+
+
+class PairItem(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("kind", "n_sides", "qx", "qy0", "qy1", "n_rows0", "n_rows1", "step_begin", "step_count",
+                 "n_loads", "partial_slot0", "partial_slot1")]
 
 
 _lock = threading.Lock()
@@ -82,6 +94,10 @@ def load() -> ctypes.CDLL:
                                           ctypes.POINTER(ctypes.POINTER(KvTile)), ctypes.POINTER(ctypes.c_int32),
                                           ctypes.POINTER(ctypes.POINTER(ctypes.c_int32)),
                                           ctypes.POINTER(ctypes.c_int32)]
+        lib.clear_plan_pair_tables.argtypes = [vp, ctypes.POINTER(ctypes.POINTER(PairItem)),
+                                               ctypes.POINTER(ctypes.c_int32),
+                                               ctypes.POINTER(ctypes.POINTER(PairStep)),
+                                               ctypes.POINTER(ctypes.c_int32)]
         lib.clear_attn_fwd_planned.argtypes = [vp, vp, vp, vp, vp, f32, vp]
         lib.clear_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, f32, vp]
         lib.clear_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
@@ -192,6 +208,14 @@ class Plan:
                                         ctypes.byref(nt), ctypes.byref(hw), ctypes.byref(nh)), "clear_plan_tables")
         return ([items[i] for i in range(ni.value)], [tiles[i] for i in range(nt.value)],
                 [hw[i] for i in range(nh.value)])
+
+    def pair_tables(self):
+        """(pair items, steps) of a TCGEN05_WS plan as lists of ctypes structs (copies)."""
+        items, steps = ctypes.POINTER(PairItem)(), ctypes.POINTER(PairStep)()
+        ni, ns = ctypes.c_int32(), ctypes.c_int32()
+        _check(load().clear_plan_pair_tables(self._h, ctypes.byref(items), ctypes.byref(ni), ctypes.byref(steps),
+                                             ctypes.byref(ns)), "clear_plan_pair_tables")
+        return [items[i] for i in range(ni.value)], [steps[i] for i in range(ns.value)]
 
     def forward(self, q, k, v, out, scale, stream=None):
         ptrs = _tensor_args(q, k, v, out, self.dtype)

@@ -18,7 +18,7 @@ namespace {
 int select_kernel(const Shape &s)
 {
     if (s.kernel != CLEAR_KERNEL_AUTO) return s.kernel;
-    if (s.dtype == CLEAR_BF16 && (s.head_dim == 64 || s.head_dim == 128)) return CLEAR_KERNEL_TCGEN05;
+    if (s.dtype == CLEAR_BF16 && (s.head_dim == 64 || s.head_dim == 128)) return CLEAR_KERNEL_TCGEN05_WS;
     return CLEAR_KERNEL_SIMT;
 }
 
@@ -44,6 +44,8 @@ int free_device_parts(clear_plan *p)
     rel(p->d_half_width);
     rel(p->d_items);
     rel(p->d_tiles);
+    rel(p->d_pair_items);
+    rel(p->d_pair_steps);
     rel(p->d_status);
     rel(p->d_partial_o);
     rel(p->d_partial_ml);
@@ -54,6 +56,8 @@ int free_device_parts(clear_plan *p)
     p->d_half_width = nullptr;
     p->d_items = nullptr;
     p->d_tiles = nullptr;
+    p->d_pair_items = nullptr;
+    p->d_pair_steps = nullptr;
     p->d_status = nullptr;
     p->d_partial_o = nullptr;
     p->d_partial_ml = nullptr;
@@ -81,12 +85,14 @@ int create_plan(clear_plan_t **out, const Shape &shape_in, bool host_only)
     try {
         if (kernel == CLEAR_KERNEL_TCGEN05)
             build_tile_schedule(s, p->sch);
+        else if (kernel == CLEAR_KERNEL_TCGEN05_WS)
+            build_pair_schedule(s, p->sch);
         else
             build_geometry(s, p->sch);
     } catch (const std::bad_alloc &) {
         return CLEAR_ERR_NO_MEMORY;
     }
-    if (kernel == CLEAR_KERNEL_TCGEN05 && p->sch.n_partial_slots > 0) {
+    if (kernel != CLEAR_KERNEL_SIMT && p->sch.n_partial_slots > 0) {
         const int64_t rows = (int64_t)s.B * s.H * p->sch.n_partial_slots * kTileTokens;
         p->workspace_bytes = rows * (s.head_dim + 2) * (int64_t)sizeof(float);
     }
@@ -95,9 +101,11 @@ int create_plan(clear_plan_t **out, const Shape &shape_in, bool host_only)
         rc = upload(&p->d_half_width, p->sch.half_width);
         if (rc == CLEAR_OK) rc = upload(&p->d_items, p->sch.items);
         if (rc == CLEAR_OK) rc = upload(&p->d_tiles, p->sch.tiles);
+        if (rc == CLEAR_OK) rc = upload(&p->d_pair_items, p->sch.pair_items);
+        if (rc == CLEAR_OK) rc = upload(&p->d_pair_steps, p->sch.pair_steps);
         if (rc == CLEAR_OK) {
-            cudaError_t e = cudaMalloc((void **)&p->d_status, sizeof(int));
-            if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
+            cudaError_t e = cudaMalloc((void **)&p->d_status, kStatusWords * sizeof(int));
+            if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, kStatusWords * sizeof(int));
             if (e != cudaSuccess) {
                 note_cuda_error((int)e);
                 (void)cudaGetLastError();
@@ -143,6 +151,7 @@ int forward(const clear_plan *p, const void *q, const void *k, const void *v, vo
     if (dev != p->device) return CLEAR_ERR_PLAN_MISMATCH;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (p->kernel == CLEAR_KERNEL_TCGEN05) return launch_tc(*p, q, k, v, out, scale, st);
+    if (p->kernel == CLEAR_KERNEL_TCGEN05_WS) return launch_ws(*p, q, k, v, out, scale, st);
     return launch_simt(*p, q, k, v, out, scale, st);
 }
 
@@ -233,6 +242,17 @@ int clear_plan_tables(const clear_plan_t *plan, const clear_work_item_t **items,
     return CLEAR_OK;
 }
 
+int clear_plan_pair_tables(const clear_plan_t *plan, const clear_pair_item_t **items, int32_t *n_items,
+                           const clear_pair_step_t **steps, int32_t *n_steps)
+{
+    if (!plan) return CLEAR_ERR_INVALID_ARG;
+    if (items) *items = plan->sch.pair_items.data();
+    if (n_items) *n_items = (int32_t)plan->sch.pair_items.size();
+    if (steps) *steps = plan->sch.pair_steps.data();
+    if (n_steps) *n_steps = (int32_t)plan->sch.pair_steps.size();
+    return CLEAR_OK;
+}
+
 int clear_attn_fwd_planned(const clear_plan_t *plan, const void *q, const void *k, const void *v, void *out,
                            float scale, void *stream)
 {
@@ -286,10 +306,11 @@ int clear_plan_info(const clear_plan_t *plan, clear_plan_info_t *info)
     info->dtype = s.dtype;
     info->kernel = plan->kernel;
     info->radius_sq_ceil = (int32_t)plan->sch.thr;
-    const bool tc = plan->kernel == CLEAR_KERNEL_TCGEN05;
+    const bool tc = plan->kernel != CLEAR_KERNEL_SIMT;
     info->tile_h = tc ? kTileH : 0;
     info->tile_w = tc ? kTileW : 0;
-    info->n_work_items = (int32_t)plan->sch.items.size();
+    info->n_work_items = plan->kernel == CLEAR_KERNEL_TCGEN05_WS ? (int32_t)plan->sch.pair_items.size()
+                                                                  : (int32_t)plan->sch.items.size();
     info->n_text_splits = plan->sch.n_text_splits;
     info->max_item_tiles = plan->sch.max_item_tiles;
     info->sum_mask = plan->sch.sum_mask;
@@ -308,7 +329,8 @@ int clear_plan_check(clear_plan_t *plan, void *stream)
     CLEAR_CUDA_TRY(cudaMemcpyAsync(&status, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost, cs));
     CLEAR_CUDA_TRY(cudaStreamSynchronize(cs));
     if (status != 0) {
-        CLEAR_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(int), cs));
+        // a block that gave up may have left the work queue of the persistent kernel mid-way
+        CLEAR_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, kStatusWords * sizeof(int), cs));
         CLEAR_CUDA_TRY(cudaStreamSynchronize(cs));
         return CLEAR_ERR_DEVICE_TIMEOUT;
     }

@@ -19,7 +19,12 @@ struct clear_plan {
     int32_t *d_half_width = nullptr;
     clear_work_item_t *d_items = nullptr;
     clear_kv_tile_t *d_tiles = nullptr;
-    int *d_status = nullptr;  // 0 = fine; set by a kernel whose bounded wait expired
+    clear_pair_item_t *d_pair_items = nullptr;
+    clear_pair_step_t *d_pair_steps = nullptr;
+    // [0] status word: 0 = fine, set by a kernel whose bounded wait expired;
+    // [1] work-queue head and [2] finished-block count of the persistent kernel (both back at zero
+    // when a launch ends)
+    int *d_status = nullptr;
 
     // split-KV workspace of the text-query rows (owned): per (bh, slot) 128 x head_dim fp32
     // un-normalised outputs, and per row the running maximum (log2 units) and the row sum
@@ -56,5 +61,11 @@ int launch_simt(const clear_plan &p, const void *q, const void *k, const void *v
                 cudaStream_t stream);
 int launch_tc(const clear_plan &p, const void *q, const void *k, const void *v, void *out, float scale,
               cudaStream_t stream);
+int launch_ws(const clear_plan &p, const void *q, const void *k, const void *v, void *out, float scale,
+              cudaStream_t stream);
+// Merge of the split-KV partial results of the text-query rows (both tensor-core kernels).
+int launch_text_combine(const clear_plan &p, void *out, cudaStream_t stream);
+
+constexpr int kStatusWords = 4;
 
 }  // namespace clear

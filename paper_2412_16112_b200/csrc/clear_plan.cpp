@@ -22,7 +22,7 @@ int validate_shape(const Shape &s)
         return CLEAR_ERR_INVALID_ARG;
     if (!(s.radius > 0.f) || !std::isfinite(s.radius)) return CLEAR_ERR_INVALID_ARG;
     if (s.dtype != CLEAR_BF16 && s.dtype != CLEAR_F32) return CLEAR_ERR_INVALID_ARG;
-    if (s.kernel < CLEAR_KERNEL_AUTO || s.kernel > CLEAR_KERNEL_TCGEN05) return CLEAR_ERR_INVALID_ARG;
+    if (s.kernel < CLEAR_KERNEL_AUTO || s.kernel > CLEAR_KERNEL_TCGEN05_WS) return CLEAR_ERR_INVALID_ARG;
     const int64_t n = (int64_t)s.grid_h * s.grid_w;
     const int64_t N = n + s.n_text;
     if (N > (int64_t)1 << 30) return CLEAR_ERR_UNSUPPORTED;  // token indices stay in int32
@@ -31,7 +31,7 @@ int validate_shape(const Shape &s)
     // 16-byte rows keep every per-token vector access and TMA stride aligned
     const int esz = s.dtype == CLEAR_BF16 ? 2 : 4;
     if ((s.head_dim * esz) % 16 != 0) return CLEAR_ERR_UNSUPPORTED;
-    if (s.kernel == CLEAR_KERNEL_TCGEN05) {
+    if (s.kernel == CLEAR_KERNEL_TCGEN05 || s.kernel == CLEAR_KERNEL_TCGEN05_WS) {
         if (s.dtype != CLEAR_BF16) return CLEAR_ERR_UNSUPPORTED;
         if (s.head_dim != 64 && s.head_dim != 128) return CLEAR_ERR_UNSUPPORTED;
     }
@@ -163,6 +163,194 @@ void build_tile_schedule(const Shape &s, Schedule &sch)
     for (const auto &it : sch.items) {
         sch.max_item_tiles = std::max(sch.max_item_tiles, it.tile_count);
         sch.executed_pairs += (int64_t)it.tile_count * kTileTokens * kTileTokens;
+    }
+}
+
+// ---- pair schedule of the warp-specialised kernel ------------------------------------------------
+namespace {
+
+struct PatchTile {
+    int x, y;
+    bool masked;
+};
+
+// Key patches (on the 8 x 16 lattice) that hold at least one key allowed to some query of the patch
+// at (qx, qy), each with the flag "some pair of the tile is not allowed".
+std::vector<PatchTile> patches_of(const Shape &s, int64_t thr, int R, int qx, int qy)
+{
+    const int gh = s.grid_h, gw = s.grid_w;
+    const int ntx = (gw + kTileW - 1) / kTileW, nty = (gh + kTileH - 1) / kTileH;
+    const int tx = qx / kTileW, ty = qy / kTileH;
+    const int reach_x = R / kTileW + 1, reach_y = R / kTileH + 1;
+    const int qx1 = std::min(qx + kTileW - 1, gw - 1), qy1 = std::min(qy + kTileH - 1, gh - 1);
+    std::vector<PatchTile> out;
+    for (int j = std::max(0, ty - reach_y); j <= std::min(nty - 1, ty + reach_y); ++j) {
+        for (int i = std::max(0, tx - reach_x); i <= std::min(ntx - 1, tx + reach_x); ++i) {
+            const int bx = i * kTileW, by = j * kTileH;
+            const int kx1 = std::min(bx + kTileW - 1, gw - 1), ky1 = std::min(by + kTileH - 1, gh - 1);
+            const int64_t gx = std::max({0, bx - qx1, qx - kx1});
+            const int64_t gy = std::max({0, by - qy1, qy - ky1});
+            if (gx * gx + gy * gy >= thr) continue;
+            const int64_t fx = std::max(kx1 - qx, qx1 - bx);
+            const int64_t fy = std::max(ky1 - qy, qy1 - by);
+            const bool whole = (bx + kTileW <= gw) && (by + kTileH <= gh);
+            out.push_back(PatchTile{bx, by, !(whole && fx * fx + fy * fy < thr)});
+        }
+    }
+    return out;
+}
+
+}  // namespace
+
+void build_pair_schedule(const Shape &s, Schedule &sch)
+{
+    build_geometry(s, sch);
+    const int gh = s.grid_h, gw = s.grid_w, T = s.n_text;
+    const int64_t N = (int64_t)gh * gw + T;
+    const int64_t thr = sch.thr;
+    const int R = (int)isqrt64(thr - 1);
+
+    sch.pair_items.clear();
+    sch.pair_steps.clear();
+
+    auto finish_item = [&](clear_pair_item_t &it) {
+        int32_t loads = 0;
+        for (int32_t i = it.step_begin; i < (int32_t)sch.pair_steps.size(); ++i) {
+            clear_pair_step_t &st = sch.pair_steps[(size_t)i];
+            st.load_base = loads;
+            const int a = (st.flags & CLEAR_STEP_USE0) ? 1 : 0;
+            const int b = ((st.flags & CLEAR_STEP_USE1) && !(st.flags & CLEAR_STEP_SHARED)) ? 1 : 0;
+            loads += 2 * (a + b);
+        }
+        it.step_count = (int32_t)sch.pair_steps.size() - it.step_begin;
+        it.n_loads = loads;
+        sch.pair_items.push_back(it);
+    };
+    auto linear_step = [&](int x, int n_valid, int n_sides) {
+        clear_pair_step_t st{};
+        st.x0 = st.x1 = x;
+        st.n_valid0 = st.n_valid1 = n_valid;
+        st.flags = CLEAR_STEP_LINEAR | CLEAR_STEP_USE0;
+        if (n_valid < kTileTokens) st.flags |= CLEAR_STEP_MASKED0;
+        if (n_sides == 2) {
+            st.flags |= CLEAR_STEP_USE1 | CLEAR_STEP_SHARED;
+            if (n_valid < kTileTokens) st.flags |= CLEAR_STEP_MASKED1;
+        }
+        sch.pair_steps.push_back(st);
+    };
+
+    // ---- text-query tiles, two per item, dense over all N keys, split over key ranges ----------
+    const int n_lin = (int)((N + kTileTokens - 1) / kTileTokens);
+    sch.n_text_tiles = (T + kTileTokens - 1) / kTileTokens;
+    int chunk = n_lin, n_splits = 1;
+    if (sch.n_text_tiles > 0) {
+        n_splits = (n_lin + kSplitTargetTiles - 1) / kSplitTargetTiles;
+        chunk = (n_lin + n_splits - 1) / n_splits;
+        n_splits = (n_lin + chunk - 1) / chunk;
+    }
+    sch.n_text_splits = sch.n_text_tiles > 0 ? n_splits : 0;
+    sch.n_partial_slots = (sch.n_text_tiles > 0 && n_splits > 1) ? sch.n_text_tiles * n_splits : 0;
+    // key range outermost: the items that stream one key range sit next to each other in the queue
+    for (int sp = 0; sp < n_splits && sch.n_text_tiles > 0; ++sp) {
+        for (int tq = 0; tq < sch.n_text_tiles; tq += 2) {
+            clear_pair_item_t it{};
+            it.kind = 1;
+            it.n_sides = (tq + 1 < sch.n_text_tiles) ? 2 : 1;
+            it.qx = tq * kTileTokens;
+            it.n_rows0 = std::min(kTileTokens, T - it.qx);
+            it.n_rows1 = it.n_sides == 2 ? std::min(kTileTokens, T - it.qx - kTileTokens) : 0;
+            it.step_begin = (int32_t)sch.pair_steps.size();
+            const int t0 = sp * chunk, t1 = std::min(n_lin, t0 + chunk);
+            for (int t = t0; t < t1; ++t)
+                linear_step(t * kTileTokens, (int)std::min<int64_t>(kTileTokens, N - (int64_t)t * kTileTokens),
+                            it.n_sides);
+            it.partial_slot0 = n_splits > 1 ? tq * n_splits + sp : -1;
+            it.partial_slot1 = (n_splits > 1 && it.n_sides == 2) ? (tq + 1) * n_splits + sp : -1;
+            finish_item(it);
+        }
+    }
+    sch.n_text_pair_items = (int)sch.pair_items.size();
+
+    // ---- image-query patches, two vertically adjacent ones per item ----------------------------
+    const int ntx = (gw + kTileW - 1) / kTileW, nty = (gh + kTileH - 1) / kTileH;
+    for (int ty = 0; ty < nty; ty += 2) {
+        for (int tx = 0; tx < ntx; ++tx) {
+            clear_pair_item_t it{};
+            it.kind = 0;
+            it.n_sides = (ty + 1 < nty) ? 2 : 1;
+            it.qx = tx * kTileW;
+            it.qy0 = ty * kTileH;
+            it.qy1 = it.qy0 + kTileH;
+            const int w = std::min(kTileW, gw - it.qx);
+            it.n_rows0 = w * std::min(kTileH, gh - it.qy0);
+            it.n_rows1 = it.n_sides == 2 ? w * std::min(kTileH, gh - it.qy1) : 0;
+            it.partial_slot0 = it.partial_slot1 = -1;
+            it.step_begin = (int32_t)sch.pair_steps.size();
+            // text keys: tokens past n_text in the last tile are image keys, not allowed through it
+            for (int t0 = 0; t0 < T; t0 += kTileTokens) linear_step(t0, std::min(kTileTokens, T - t0), it.n_sides);
+
+            std::vector<PatchTile> a = patches_of(s, thr, R, it.qx, it.qy0), b;
+            if (it.n_sides == 2) b = patches_of(s, thr, R, it.qx, it.qy1);
+            auto find = [](const std::vector<PatchTile> &v, const PatchTile &t) -> const PatchTile * {
+                for (const PatchTile &u : v)
+                    if (u.x == t.x && u.y == t.y) return &u;
+                return nullptr;
+            };
+            std::vector<PatchTile> only_a, only_b;
+            std::vector<std::pair<PatchTile, PatchTile>> both;
+            for (const PatchTile &t : a) {
+                const PatchTile *u = find(b, t);
+                if (u)
+                    both.push_back({t, *u});
+                else
+                    only_a.push_back(t);
+            }
+            for (const PatchTile &t : b)
+                if (!find(a, t)) only_b.push_back(t);
+            // key patches only one tile needs are taken two at a time, one per tile, so that both
+            // tiles stay busy; what is left over runs one-sided
+            for (size_t i = 0; i < std::max(only_a.size(), only_b.size()); ++i) {
+                clear_pair_step_t st{};
+                st.n_valid0 = st.n_valid1 = kTileTokens;
+                if (i < only_a.size()) {
+                    st.x0 = only_a[i].x;
+                    st.y0 = only_a[i].y;
+                    st.flags |= CLEAR_STEP_USE0 | (only_a[i].masked ? CLEAR_STEP_MASKED0 : 0);
+                }
+                if (i < only_b.size()) {
+                    st.x1 = only_b[i].x;
+                    st.y1 = only_b[i].y;
+                    st.flags |= CLEAR_STEP_USE1 | (only_b[i].masked ? CLEAR_STEP_MASKED1 : 0);
+                }
+                sch.pair_steps.push_back(st);
+            }
+            for (const auto &ab : both) {
+                clear_pair_step_t st{};
+                st.n_valid0 = st.n_valid1 = kTileTokens;
+                st.x0 = st.x1 = ab.first.x;
+                st.y0 = st.y1 = ab.first.y;
+                st.flags = CLEAR_STEP_USE0 | CLEAR_STEP_USE1 | CLEAR_STEP_SHARED |
+                           (ab.first.masked ? CLEAR_STEP_MASKED0 : 0) | (ab.second.masked ? CLEAR_STEP_MASKED1 : 0);
+                sch.pair_steps.push_back(st);
+            }
+            finish_item(it);
+        }
+    }
+
+    // ---- work order: text items (the longest lists) first, then image items, longest first; the
+    // blocks take items from the queue in this order, so the short border items fill the tail
+    std::stable_sort(sch.pair_items.begin() + sch.n_text_pair_items, sch.pair_items.end(),
+                     [](const clear_pair_item_t &x, const clear_pair_item_t &y) { return x.step_count > y.step_count; });
+
+    sch.max_item_tiles = 0;
+    sch.executed_pairs = 0;
+    for (const auto &it : sch.pair_items) {
+        sch.max_item_tiles = std::max(sch.max_item_tiles, it.step_count);
+        for (int32_t i = 0; i < it.step_count; ++i) {
+            const int f = sch.pair_steps[(size_t)(it.step_begin + i)].flags;
+            const int uses = ((f & CLEAR_STEP_USE0) ? 1 : 0) + ((f & CLEAR_STEP_USE1) ? 1 : 0);
+            sch.executed_pairs += (int64_t)uses * kTileTokens * kTileTokens;
+        }
     }
 }
 

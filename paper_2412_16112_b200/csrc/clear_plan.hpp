@@ -30,6 +30,9 @@ struct Schedule {
     std::vector<int32_t> half_width;     // half_width[dy] = max |dx| allowed at row offset dy
     std::vector<clear_work_item_t> items;
     std::vector<clear_kv_tile_t> tiles;
+    std::vector<clear_pair_item_t> pair_items;   // TCGEN05_WS: text items first, then image items
+    std::vector<clear_pair_step_t> pair_steps;
+    int n_text_pair_items = 0;
     int n_text_tiles = 0;                // text-query tiles of 128 rows
     int n_text_splits = 0;               // splits per text-query tile (1 = no partial results)
     int n_partial_slots = 0;
@@ -46,5 +49,8 @@ void build_geometry(const Shape &s, Schedule &sch);
 
 // Work items and key-tile lists of the tensor-core kernel (calls build_geometry first).
 void build_tile_schedule(const Shape &s, Schedule &sch);
+
+// Pair items and step lists of the warp-specialised tensor-core kernel (calls build_geometry first).
+void build_pair_schedule(const Shape &s, Schedule &sch);
 
 }  // namespace clear

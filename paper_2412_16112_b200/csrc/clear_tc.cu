@@ -530,17 +530,28 @@ int launch_variant(const clear_plan &p, const CUtensorMap *tm, const TcParams &p
     clear_tc_kernel<D, P_SMEM><<<grid, kThreads, kSmem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], tm[7],
                                                                   prm);
     CLEAR_CUDA_TRY(cudaGetLastError());
-    if (p.sch.n_partial_slots > 0) {
-        const int64_t N = (int64_t)s.n_text + (int64_t)s.grid_h * s.grid_w;
-        dim3 cgrid((unsigned)s.n_text, (unsigned)(s.B * s.H));
-        clear_tc_combine_kernel<D><<<cgrid, D, 0, stream>>>(p.d_partial_o, p.d_partial_ml, (__nv_bfloat16 *)out, s.n_text,
-                                                            N, p.sch.n_text_splits, p.sch.n_partial_slots);
-        CLEAR_CUDA_TRY(cudaGetLastError());
-    }
-    return CLEAR_OK;
+    return launch_text_combine(p, out, stream);
 }
 
 }  // namespace
+
+int launch_text_combine(const clear_plan &p, void *out, cudaStream_t stream)
+{
+    const Shape &s = p.shape;
+    if (p.sch.n_partial_slots <= 0) return CLEAR_OK;
+    const int64_t N = (int64_t)s.n_text + (int64_t)s.grid_h * s.grid_w;
+    dim3 cgrid((unsigned)s.n_text, (unsigned)(s.B * s.H));
+    if (s.head_dim == 128)
+        clear_tc_combine_kernel<128><<<cgrid, 128, 0, stream>>>(p.d_partial_o, p.d_partial_ml, (__nv_bfloat16 *)out,
+                                                                s.n_text, N, p.sch.n_text_splits, p.sch.n_partial_slots);
+    else if (s.head_dim == 64)
+        clear_tc_combine_kernel<64><<<cgrid, 64, 0, stream>>>(p.d_partial_o, p.d_partial_ml, (__nv_bfloat16 *)out,
+                                                              s.n_text, N, p.sch.n_text_splits, p.sch.n_partial_slots);
+    else
+        return CLEAR_ERR_UNSUPPORTED;
+    CLEAR_CUDA_TRY(cudaGetLastError());
+    return CLEAR_OK;
+}
 
 int launch_tc(const clear_plan &p, const void *q, const void *k, const void *v, void *out, float scale,
               cudaStream_t stream)

@@ -1,0 +1,809 @@
+// CLEAR attention forward on the sm_100a tensor cores: persistent, warp-specialised kernel.
+//
+// One thread block per SM takes work items from a queue (an atomic counter).  A work item is a PAIR
+// of 128-query tiles -- two vertically adjacent 8 x 16 patches of the latent grid, or two tiles of
+// text tokens -- and a list of steps; in each step every query tile of the pair meets one 128-key
+// tile (Eq. 1 restricted by Eq. 3).  Key tiles both query tiles need are staged once.
+//
+// Roles (512 threads):
+//   warp 0        : takes items from the queue and issues every TMA load (Q tiles, K/V ring);
+//   warp 1        : issues every tcgen05.mma: S_t = Q_t K^T, O_t += P_t V, t = 0, 1, interleaved so
+//                   that the softmax of one query tile runs under the MMAs of the other;
+//   warps 4-7     : softmax of query tile 0 (thread r owns query row r = tensor-memory lane r):
+//                   mask, running maximum, P = exp2(.), row sum, P (bf16) back into tensor memory;
+//   warps 8-11    : the same for query tile 1;
+//   warps 12-15   : epilogue: O / l -> bf16 -> global memory (or fp32 partial results of split
+//                   text rows), while the other warps already run the next item.
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each; P overwrites S in place.
+// Shared memory: Q0, Q1 and a ring of five key/value stages (K and V tiles take one stage each).
+// Every wait is bounded: on expiry the block raises the plan's status word and leaves.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstring>
+
+#include "clear_internal.hpp"
+#include "ptx.cuh"
+
+namespace clear {
+namespace {
+
+constexpr int kWsThreads = 512;
+constexpr int kRing = 5;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the row max grows by more
+constexpr int kSchedDepth = 2;
+// arrivals that free a queue slot: the MMA thread and one lane of each of the 12 softmax / epilogue warps
+constexpr uint32_t kSchedReaders = 13;
+// registers per thread of each role (warpgroups of 128 threads: 48 + 2 * 192 + 80 = 512)
+constexpr uint32_t kRegsControl = 48, kRegsSoftmax = 192, kRegsEpilogue = 80;
+
+struct WsParams {
+    const clear_pair_item_t *items;
+    const clear_pair_step_t *steps;
+    const int32_t *half_width;
+    int n_half_width;
+    int grid_h, grid_w, n_text;
+    long long n_tokens;
+    int n_items, n_text_items, n_bh;
+    float scale_log2;  // scale * log2(e)
+    float *partial_o;
+    float *partial_ml;
+    int n_partial_slots;
+    __nv_bfloat16 *out;
+    int *status;  // [0] status word, [1] queue head, [2] finished blocks
+};
+
+struct Ctrl {
+    uint64_t q_full[2], q_empty[2];
+    uint64_t kv_full[kRing], kv_empty[kRing];
+    uint64_t s_full[2], p_ready[2], o_full[2], o_empty[2], stats_full[2], stats_empty[2];
+    uint64_t sched_full[kSchedDepth], sched_empty[kSchedDepth];
+    uint64_t drain;
+    int32_t sched_item[kSchedDepth];
+    uint32_t tmem_base;
+    int abort_flag;
+    int skip;
+    float2 stats[2][128];  // per query row: running maximum (log2 units) and row sum
+};
+
+// Bounded wait on an mbarrier phase.  Returns false once the block has given up.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (it > 256) __nanosleep(it > 8192 ? 256 : 32);
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicExch(status, code);
+    return false;
+}
+// Drain: wait for a phase regardless of the abort flag (used before leaving with copies in flight).
+__device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (ptx::mbar_try_wait(bar, parity)) return;
+        if (it > 64) __nanosleep(256);
+    }
+}
+
+struct ItemRef {
+    int bh;
+    int item;
+};
+// Queue position -> (batch*head, item): every text item of every head first, then the image items.
+__device__ __forceinline__ ItemRef decode_item(const WsParams &prm, int g)
+{
+    ItemRef r;
+    const int n_txt_all = prm.n_text_items * prm.n_bh;
+    if (g < n_txt_all) {
+        r.bh = g / prm.n_text_items;
+        r.item = g - r.bh * prm.n_text_items;
+    } else {
+        const int n_img = prm.n_items - prm.n_text_items;
+        const int g2 = g - n_txt_all;
+        r.bh = g2 / n_img;
+        r.item = prm.n_text_items + (g2 - r.bh * n_img);
+    }
+    return r;
+}
+
+__device__ __forceinline__ clear_pair_step_t load_step(const clear_pair_step_t *p)
+{
+    const int4 a = __ldg(reinterpret_cast<const int4 *>(p));
+    const int4 b = __ldg(reinterpret_cast<const int4 *>(p) + 1);
+    clear_pair_step_t s;
+    s.x0 = a.x; s.y0 = a.y; s.x1 = a.z; s.y1 = a.w;
+    s.flags = b.x; s.n_valid0 = b.y; s.n_valid1 = b.z; s.load_base = b.w;
+    return s;
+}
+__device__ __forceinline__ clear_pair_item_t load_item(const clear_pair_item_t *p)
+{
+    const int4 a = __ldg(reinterpret_cast<const int4 *>(p));
+    const int4 b = __ldg(reinterpret_cast<const int4 *>(p) + 1);
+    const int4 c = __ldg(reinterpret_cast<const int4 *>(p) + 2);
+    clear_pair_item_t it;
+    it.kind = a.x; it.n_sides = a.y; it.qx = a.z; it.qy0 = a.w;
+    it.qy1 = b.x; it.n_rows0 = b.y; it.n_rows1 = b.z; it.step_begin = b.w;
+    it.step_count = c.x; it.n_loads = c.y; it.partial_slot0 = c.z; it.partial_slot1 = c.w;
+    return it;
+}
+static_assert(sizeof(clear_pair_step_t) == 32 && sizeof(clear_pair_item_t) == 48, "table records are read as int4");
+
+__device__ __forceinline__ bool step_uses(int flags, int side) { return (flags & (side ? CLEAR_STEP_USE1 : CLEAR_STEP_USE0)) != 0; }
+// Ring positions (relative to the step's load_base) of the K and V tiles a side reads in a step:
+// stages are filled in the order K(tile 0), K(tile 1), V(tile 0), V(tile 1), skipping what is absent.
+__device__ __forceinline__ int step_n_tiles(int flags)
+{
+    const int a = (flags & CLEAR_STEP_USE0) ? 1 : 0;
+    const int b = ((flags & CLEAR_STEP_USE1) && !(flags & CLEAR_STEP_SHARED)) ? 1 : 0;
+    return a + b;
+}
+__device__ __forceinline__ int step_tile_index(int flags, int side)
+{
+    if (side == 0 || (flags & CLEAR_STEP_SHARED)) return 0;
+    return (flags & CLEAR_STEP_USE0) ? 1 : 0;
+}
+// Is `side` the last reader of its tile in this step?  (Tile 1 runs after tile 0 within a step.)
+__device__ __forceinline__ bool step_last_reader(int flags, int side)
+{
+    if (!(flags & CLEAR_STEP_SHARED)) return true;
+    return side == 1;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kWsThreads, 1)
+clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_constant__ CUtensorMap tm_k_img,
+                const __grid_constant__ CUtensorMap tm_v_img, const __grid_constant__ CUtensorMap tm_q_txt,
+                const __grid_constant__ CUtensorMap tm_k_lin, const __grid_constant__ CUtensorMap tm_v_lin,
+                const WsParams prm)
+{
+    constexpr int kHalves = D / 64;                 // 64-channel (128-byte) column blocks of a tile
+    constexpr uint32_t kHalfBytes = 128 * 128;      // 128 rows x 128 B
+    constexpr uint32_t kTileBytes = kHalves * kHalfBytes;
+    constexpr uint32_t kIdescQK = ptx::idesc_bf16(128, false);
+    constexpr uint32_t kIdescPV = ptx::idesc_bf16(D, true);
+
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t smem_base = ptx::smem_u32(smem_raw);
+    const uint32_t sQ = smem_base, sRing = sQ + 2 * kTileBytes;
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_raw + (2 + kRing) * kTileBytes);
+    volatile int *abort_flag = &ctrl->abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int total_items = prm.n_items * prm.n_bh;
+
+    // once any block of this launch has given up, the rest of the grid leaves at once; a window that
+    // is not 1024-byte aligned (never expected) cannot hold swizzled tiles
+    if (tid == 0) {
+        int skip = *reinterpret_cast<volatile int *>(prm.status);
+        if ((smem_base & 1023u) != 0u) {
+            atomicExch(prm.status, 100);
+            skip = 1;
+        }
+        ctrl->skip = skip;
+    }
+    __syncthreads();
+    if (ctrl->skip != 0) {
+        if (tid == 0) {
+            // keep the finished-block count right so that the queue is reset for the next launch
+            const int done = atomicAdd(prm.status + 2, 1);
+            if (done == (int)gridDim.x - 1) {
+                atomicExch(prm.status + 1, 0);
+                atomicExch(prm.status + 2, 0);
+            }
+        }
+        return;
+    }
+
+    if (tid == 0) {
+        ctrl->abort_flag = 0;
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&ctrl->q_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->q_empty[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->s_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->o_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->stats_full[i]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->stats_empty[i]), 128);
+        }
+        for (int i = 0; i < kRing; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&ctrl->kv_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->kv_empty[i]), 1);
+        }
+        for (int i = 0; i < kSchedDepth; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&ctrl->sched_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->sched_empty[i]), kSchedReaders);
+        }
+        ptx::mbar_init(ptx::smem_u32(&ctrl->drain), 1);
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem = ctrl->tmem_base;
+
+    if (warp < 4) {
+        ptx::setmaxnreg_dec<kRegsControl>();
+        if (warp == 0 && lane == 0) {
+            // ================= loader: work queue + every TMA load ====================================
+            uint32_t n_loads = 0;    // K/V stages filled so far by this block
+            uint32_t n_q[2] = {0, 0};
+            for (uint32_t k = 0;; ++k) {
+                const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
+                if (!wait_bar(ptx::smem_u32(&ctrl->sched_empty[slot]), (use & 1u) ^ 1u, abort_flag, prm.status, 1)) break;
+                const int g = atomicAdd(prm.status + 1, 1);
+                ctrl->sched_item[slot] = g;
+                ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_full[slot]));
+                if (g >= total_items) break;
+                const ItemRef ref = decode_item(prm, g);
+                const clear_pair_item_t item = load_item(prm.items + ref.item);
+                bool ok = true;
+                for (int t = 0; t < item.n_sides && ok; ++t) {
+                    const uint32_t bar = ptx::smem_u32(&ctrl->q_full[t]);
+                    ok = wait_bar(ptx::smem_u32(&ctrl->q_empty[t]), (n_q[t] & 1u) ^ 1u, abort_flag, prm.status, 2);
+                    if (!ok) break;
+                    ptx::mbar_expect_tx(bar, kTileBytes);
+#pragma unroll
+                    for (int h = 0; h < kHalves; ++h) {
+                        const uint32_t dst = sQ + t * kTileBytes + h * kHalfBytes;
+                        if (item.kind == 1)
+                            ptx::tma_load_3d(dst, &tm_q_txt, bar, h * 64, item.qx + t * 128, ref.bh);
+                        else
+                            ptx::tma_load_4d(dst, &tm_q_img, bar, h * 64, item.qx, t ? item.qy1 : item.qy0, ref.bh);
+                    }
+                    ++n_q[t];
+                }
+                const clear_pair_step_t *steps = prm.steps + item.step_begin;
+                for (int s = 0; s < item.step_count && ok; ++s) {
+                    const clear_pair_step_t st = load_step(steps + s);
+                    const bool has_a = (st.flags & CLEAR_STEP_USE0) != 0;
+                    const bool has_b = (st.flags & CLEAR_STEP_USE1) && !(st.flags & CLEAR_STEP_SHARED);
+                    const bool linear = (st.flags & CLEAR_STEP_LINEAR) != 0;
+#pragma unroll
+                    for (int kv = 0; kv < 2; ++kv) {
+#pragma unroll
+                        for (int t = 0; t < 2; ++t) {
+                            if (!ok || (t == 0 ? !has_a : !has_b)) continue;
+                            const uint32_t stage = n_loads % kRing, fill = n_loads / kRing;
+                            ok = wait_bar(ptx::smem_u32(&ctrl->kv_empty[stage]), (fill & 1u) ^ 1u, abort_flag, prm.status, 3);
+                            if (!ok) continue;
+                            const uint32_t bar = ptx::smem_u32(&ctrl->kv_full[stage]);
+                            const uint32_t dst = sRing + stage * kTileBytes;
+                            const int x = t ? st.x1 : st.x0, y = t ? st.y1 : st.y0;
+                            ptx::mbar_expect_tx(bar, kTileBytes);
+#pragma unroll
+                            for (int h = 0; h < kHalves; ++h) {
+                                if (linear)
+                                    ptx::tma_load_3d(dst + h * kHalfBytes, kv ? &tm_v_lin : &tm_k_lin, bar, h * 64, x, ref.bh);
+                                else
+                                    ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_v_img : &tm_k_img, bar, h * 64, x, y, ref.bh);
+                            }
+                            ++n_loads;
+                        }
+                    }
+                }
+                if (!ok) break;
+            }
+            if (*abort_flag) {
+                // leave no copy in flight: whatever was issued must land before the block exits
+                for (int t = 0; t < 2; ++t)
+                    if (n_q[t] > 0) drain_bar(ptx::smem_u32(&ctrl->q_full[t]), (n_q[t] - 1) & 1u);
+                for (uint32_t j = 0; j < (uint32_t)kRing && j < n_loads; ++j) {
+                    const uint32_t idx = n_loads - 1 - j;
+                    drain_bar(ptx::smem_u32(&ctrl->kv_full[idx % kRing]), (idx / kRing) & 1u);
+                }
+            }
+        } else if (warp == 1 && lane == 0) {
+            // ================= MMA issuer ================================================================
+            uint32_t ring_base = 0;          // K/V stages consumed by the items before this one
+            uint32_t n_q[2] = {0, 0};        // items seen per query tile
+            uint32_t n_p[2] = {0, 0};        // P tiles consumed per query tile
+            bool ok = true;
+            auto kv_wait = [&](uint32_t pos) -> uint32_t {
+                const uint32_t stage = pos % kRing, fill = pos / kRing;
+                ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[stage]), fill & 1u, abort_flag, prm.status, 4);
+                return stage;
+            };
+            for (uint32_t k = 0; ok; ++k) {
+                const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
+                if (!wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 5)) break;
+                const int g = ctrl->sched_item[slot];
+                ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
+                if (g >= total_items) break;
+                const ItemRef ref = decode_item(prm, g);
+                const clear_pair_item_t item = load_item(prm.items + ref.item);
+                const clear_pair_step_t *steps = prm.steps + item.step_begin;
+                const int n = item.step_count;
+                for (int t = 0; t < item.n_sides && ok; ++t)
+                    ok = wait_bar(ptx::smem_u32(&ctrl->q_full[t]), n_q[t] & 1u, abort_flag, prm.status, 6);
+                if (!ok) break;
+
+                // S_t = Q_t K^T for the key tile of `st`
+                auto issue_qk = [&](const clear_pair_step_t &st, int t) {
+                    const uint32_t pos = ring_base + (uint32_t)st.load_base + (uint32_t)step_tile_index(st.flags, t);
+                    const uint32_t stage = kv_wait(pos);
+                    if (!ok) return;
+                    ptx::tc_fence_after();
+                    const uint32_t sK = sRing + stage * kTileBytes, sQt = sQ + t * kTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                        ptx::mma_ss(tmem + t * 128, ptx::smem_desc_sw128(sQt + off, 16, 1024),
+                                    ptx::smem_desc_sw128(sK + off, 16, 1024), kIdescQK, kk > 0);
+                    }
+                    ptx::tc_commit(ptx::smem_u32(&ctrl->s_full[t]));
+                    if (step_last_reader(st.flags, t)) ptx::tc_commit(ptx::smem_u32(&ctrl->kv_empty[stage]));
+                };
+
+                clear_pair_step_t cur = load_step(steps);
+                for (int t = 0; t < 2 && ok; ++t)
+                    if (step_uses(cur.flags, t)) issue_qk(cur, t);
+                if (n == 1) {
+                    for (int t = 0; t < item.n_sides; ++t) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
+                }
+                uint32_t n_pv[2] = {0, 0};
+                for (int s = 0; s < n && ok; ++s) {
+                    clear_pair_step_t nxt = cur;
+                    const bool has_next = s + 1 < n;
+                    if (has_next) nxt = load_step(steps + s + 1);
+                    for (int t = 0; t < 2 && ok; ++t) {
+                        if (step_uses(cur.flags, t)) {
+                            // O_t += P_t V
+                            ok = wait_bar(ptx::smem_u32(&ctrl->p_ready[t]), n_p[t] & 1u, abort_flag, prm.status, 7);
+                            if (!ok) break;
+                            ++n_p[t];
+                            const uint32_t pos = ring_base + (uint32_t)cur.load_base + (uint32_t)step_n_tiles(cur.flags) +
+                                                 (uint32_t)step_tile_index(cur.flags, t);
+                            const uint32_t stage = kv_wait(pos);
+                            if (!ok) break;
+                            if (n_pv[t] == 0) {
+                                // the epilogue must have read the previous item's O_t out of tensor memory
+                                ok = wait_bar(ptx::smem_u32(&ctrl->o_empty[t]), (n_q[t] & 1u) ^ 1u, abort_flag, prm.status, 8);
+                                if (!ok) break;
+                            }
+                            ptx::tc_fence_after();
+                            const uint32_t sV = sRing + stage * kTileBytes;
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) {
+                                const uint64_t bdesc = ptx::smem_desc_sw128(sV + kk * 2048, kHalfBytes, 1024);
+                                ptx::mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, bdesc, kIdescPV,
+                                            (n_pv[t] > 0 || kk > 0) ? 1u : 0u);
+                            }
+                            ++n_pv[t];
+                            if (step_last_reader(cur.flags, t)) ptx::tc_commit(ptx::smem_u32(&ctrl->kv_empty[stage]));
+                        }
+                        if (!has_next && t < item.n_sides) ptx::tc_commit(ptx::smem_u32(&ctrl->o_full[t]));
+                        if (has_next && step_uses(nxt.flags, t)) issue_qk(nxt, t);
+                    }
+                    if (has_next && s + 2 == n) {
+                        // every Q_t K^T of the item has been issued: the next item's Q tiles may land
+                        for (int t = 0; t < item.n_sides; ++t) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
+                    }
+                    cur = nxt;
+                }
+                for (int t = 0; t < item.n_sides; ++t) ++n_q[t];
+                ring_base += (uint32_t)item.n_loads;
+            }
+            if (*abort_flag) {
+                // MMAs that were issued must retire before tensor memory is given back
+                ptx::tc_commit(ptx::smem_u32(&ctrl->drain));
+                drain_bar(ptx::smem_u32(&ctrl->drain), 0);
+            }
+        }
+        __syncwarp();
+    } else if (warp < 12) {
+        // ================= softmax warps: thread r owns query row r of its tile =========================
+        ptx::setmaxnreg_inc<kRegsSoftmax>();
+        const int t = (warp - 4) >> 2;           // query tile of the pair
+        const int r = tid & 127;
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
+        const float c = prm.scale_log2;
+        const uint32_t b_s = ptx::smem_u32(&ctrl->s_full[t]), b_p = ptx::smem_u32(&ctrl->p_ready[t]);
+        uint32_t n_s = 0, n_items_seen = 0;
+        bool alive = true;
+        for (uint32_t k = 0; alive; ++k) {
+            const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
+            if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 9)))
+                break;
+            const int g = ctrl->sched_item[slot];
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
+            if (g >= total_items) break;
+            const ItemRef ref = decode_item(prm, g);
+            const clear_pair_item_t item = load_item(prm.items + ref.item);
+            if (t >= item.n_sides) continue;
+            const clear_pair_step_t *steps = prm.steps + item.step_begin;
+            const bool is_text = item.kind == 1;
+            int q_y = 0, q_x = 0;
+            bool q_valid;
+            if (is_text) {
+                q_valid = r < (t ? item.n_rows1 : item.n_rows0);
+            } else {
+                q_y = (t ? item.qy1 : item.qy0) + (r >> 4);
+                q_x = item.qx + (r & 15);
+                q_valid = q_y < prm.grid_h && q_x < prm.grid_w;
+            }
+            float m_used = -INFINITY, l = 0.f;
+            bool first = true;
+
+            for (int s = 0; s < item.step_count; ++s) {
+                const clear_pair_step_t st = load_step(steps + s);
+                if (!step_uses(st.flags, t)) continue;
+                const bool masked = (st.flags & (t ? CLEAR_STEP_MASKED1 : CLEAR_STEP_MASKED0)) != 0;
+                const int k_x = t ? st.x1 : st.x0, k_y = t ? st.y1 : st.y0;
+                // ---- mask bits of this row for the tile (bit j = key j allowed) -----------------------
+                uint32_t mw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+                if (masked) {
+                    if (st.flags & CLEAR_STEP_LINEAR) {
+                        const int n_valid = t ? st.n_valid1 : st.n_valid0;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            const int nv = min(max(n_valid - 32 * w, 0), 32);
+                            mw[w] = nv == 32 ? 0xffffffffu : ((1u << nv) - 1u);
+                        }
+                    } else {
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) mw[w] = 0u;
+#pragma unroll
+                        for (int rr = 0; rr < 8; ++rr) {
+                            const int ky = k_y + rr;
+                            const int ady = abs(ky - q_y);
+                            uint32_t bits = 0u;
+                            if (q_valid && ky >= 0 && ky < prm.grid_h && ady < prm.n_half_width) {
+                                const int hw = __ldg(prm.half_width + ady);
+                                const int lo = max(max(q_x - hw, 0), k_x);
+                                const int hi = min(min(q_x + hw, prm.grid_w - 1), k_x + 15);
+                                if (lo <= hi) bits = ((1u << (hi - lo + 1)) - 1u) << (lo - k_x);
+                            }
+                            mw[rr >> 1] |= bits << (16 * (rr & 1));
+                        }
+                    }
+                }
+
+                // warp-uniform outcome: the tcgen05.ld / st below need the whole warp
+                if (!__all_sync(0xffffffffu, wait_bar(b_s, n_s & 1u, abort_flag, prm.status, 10))) {
+                    alive = false;
+                    break;
+                }
+                ++n_s;
+                ptx::tc_fence_after();
+                uint32_t sv[4][32];
+#pragma unroll
+                for (int w = 0; w < 4; ++w) ptx::tmem_ld32(tmem_S + lane_off + 32 * w, sv[w]);
+                ptx::tmem_wait_ld();
+
+                float mx = -INFINITY;
+                if (masked) {
+#pragma unroll
+                    for (int w = 0; w < 4; ++w)
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float val = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
+                            sv[w][j] = __float_as_uint(val);
+                            mx = fmaxf(mx, val);
+                        }
+                } else {
+#pragma unroll
+                    for (int w = 0; w < 4; ++w)
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(sv[w][j]));
+                }
+
+                // ---- running maximum; O is rescaled only when it grew by more than the threshold -----
+                const float m_new = fmaxf(m_used, mx);
+                if (first) {
+                    m_used = m_new;
+                    first = false;
+                } else {
+                    const bool need = (m_new - m_used) * c > kRescaleThreshold;  // false for NaN (-inf minus -inf)
+                    if (__any_sync(0xffffffffu, need)) {
+                        float alpha = 1.f;
+                        if (need) {
+                            alpha = ptx::ex2((m_used - m_new) * c);
+                            m_used = m_new;
+                            l *= alpha;
+                        }
+                        // S_t being ready means every earlier MMA, the last P_t V included, has retired
+#pragma unroll 1
+                        for (int w = 0; w < D / 16; ++w) {
+                            uint32_t o[16];
+                            ptx::tmem_ld16(tmem_O + lane_off + 16 * w, o);
+                            ptx::tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                            ptx::tmem_st16(tmem_O + lane_off + 16 * w, o);
+                        }
+                    }
+                }
+                const float mc = (m_used == -INFINITY) ? 0.f : m_used * c;
+
+                // ---- P = exp2(S * c - m * c), row sum, bf16 pairs over the first 64 columns of S -----
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        const float p0 = ptx::ex2(fmaf(__uint_as_float(sv[w][j]), c, -mc));
+                        const float p1 = ptx::ex2(fmaf(__uint_as_float(sv[w][j + 1]), c, -mc));
+                        l += p0 + p1;
+                        pk[j >> 1] = ptx::pack_bf16(p0, p1);
+                    }
+                    ptx::tmem_st16(tmem_S + lane_off + 16 * w, pk);
+                }
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(b_p);
+            }
+            if (!alive) break;
+
+            // ---- hand the row statistics to the epilogue warps ------------------------------------
+            if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->stats_empty[t]), (n_items_seen & 1u) ^ 1u, abort_flag,
+                                                  prm.status, 11)))
+                break;
+            ctrl->stats[t][r] = make_float2(m_used * c, l);
+            ptx::mbar_arrive(ptx::smem_u32(&ctrl->stats_full[t]));
+            ++n_items_seen;
+        }
+    } else {
+        // ================= epilogue warps: O_t / l -> global memory ========================================
+        ptx::setmaxnreg_dec<kRegsEpilogue>();
+        const int r = tid & 127;
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        uint32_t n_seen[2] = {0, 0};
+        bool alive = true;
+        for (uint32_t k = 0; alive; ++k) {
+            const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
+            if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 12)))
+                break;
+            const int g = ctrl->sched_item[slot];
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
+            if (g >= total_items) break;
+            const ItemRef ref = decode_item(prm, g);
+            const clear_pair_item_t item = load_item(prm.items + ref.item);
+            for (int t = 0; t < item.n_sides; ++t) {
+                const uint32_t ph = n_seen[t] & 1u;
+                if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->stats_full[t]), ph, abort_flag, prm.status, 13))) {
+                    alive = false;
+                    break;
+                }
+                const float2 ml = ctrl->stats[t][r];
+                ptx::mbar_arrive(ptx::smem_u32(&ctrl->stats_empty[t]));
+                if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->o_full[t]), ph, abort_flag, prm.status, 14))) {
+                    alive = false;
+                    break;
+                }
+                ++n_seen[t];
+                ptx::tc_fence_after();
+                const uint32_t tmem_O = tmem + 256 + t * 128;
+                // which token is row r, and does it exist?
+                long long token;
+                bool q_valid;
+                if (item.kind == 1) {
+                    token = item.qx + t * 128 + r;
+                    q_valid = r < (t ? item.n_rows1 : item.n_rows0);
+                } else {
+                    const int q_y = (t ? item.qy1 : item.qy0) + (r >> 4), q_x = item.qx + (r & 15);
+                    q_valid = q_y < prm.grid_h && q_x < prm.grid_w;
+                    token = prm.n_text + (long long)q_y * prm.grid_w + q_x;
+                }
+                const int slot_p = t ? item.partial_slot1 : item.partial_slot0;
+                if (slot_p >= 0) {
+                    // split text-query tile: un-normalised fp32 row, its maximum (log2 units) and its sum
+                    const long long row = ((long long)ref.bh * prm.n_partial_slots + slot_p) * 128 + r;
+                    float *dst = prm.partial_o + row * D;
+#pragma unroll
+                    for (int w = 0; w < D / 32; ++w) {
+                        uint32_t o[32];
+                        ptx::tmem_ld32(tmem_O + lane_off + 32 * w, o);
+                        ptx::tmem_wait_ld();
+                        if (w == D / 32 - 1) {
+                            ptx::tc_fence_before();
+                            ptx::mbar_arrive(ptx::smem_u32(&ctrl->o_empty[t]));
+                        }
+                        if (q_valid) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<uint4 *>(dst + 32 * w + j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+                        }
+                    }
+                    if (q_valid) {
+                        prm.partial_ml[row * 2] = ml.x;
+                        prm.partial_ml[row * 2 + 1] = ml.y;
+                    }
+                } else {
+                    const float inv = ml.y > 0.f ? 1.f / ml.y : 0.f;
+                    __nv_bfloat16 *dst = prm.out + ((long long)ref.bh * prm.n_tokens + token) * D;
+#pragma unroll
+                    for (int w = 0; w < D / 32; ++w) {
+                        uint32_t o[32];
+                        ptx::tmem_ld32(tmem_O + lane_off + 32 * w, o);
+                        ptx::tmem_wait_ld();
+                        if (w == D / 32 - 1) {
+                            ptx::tc_fence_before();
+                            ptx::mbar_arrive(ptx::smem_u32(&ctrl->o_empty[t]));
+                        }
+                        if (q_valid) {
+#pragma unroll
+                            for (int cc = 0; cc < 4; ++cc) {
+                                uint4 val;
+                                val.x = ptx::pack_bf16(__uint_as_float(o[8 * cc + 0]) * inv, __uint_as_float(o[8 * cc + 1]) * inv);
+                                val.y = ptx::pack_bf16(__uint_as_float(o[8 * cc + 2]) * inv, __uint_as_float(o[8 * cc + 3]) * inv);
+                                val.z = ptx::pack_bf16(__uint_as_float(o[8 * cc + 4]) * inv, __uint_as_float(o[8 * cc + 5]) * inv);
+                                val.w = ptx::pack_bf16(__uint_as_float(o[8 * cc + 6]) * inv, __uint_as_float(o[8 * cc + 7]) * inv);
+                                *reinterpret_cast<uint4 *>(dst + 32 * w + 8 * cc) = val;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, kTmemCols);
+    }
+    if (tid == 0) {
+        // the last block to finish puts the queue back to zero for the next launch
+        const int done = atomicAdd(prm.status + 2, 1);
+        if (done == (int)gridDim.x - 1) {
+            atomicExch(prm.status + 1, 0);
+            atomicExch(prm.status + 2, 0);
+        }
+    }
+}
+
+// ---- host side: tensor maps and launch ---------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// bf16 tensor of `rank` dims (innermost first); strides in bytes for dims 1..rank-1.
+bool encode(CUtensorMap *tm, const void *base, int rank, const uint64_t *dims, const uint64_t *strides,
+            const uint32_t *box)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base),
+                     reinterpret_cast<const cuuint64_t *>(dims), reinterpret_cast<const cuuint64_t *>(strides),
+                     reinterpret_cast<const cuuint32_t *>(box), ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS;
+}
+
+// Maps 0..2: image part of q, k, v as [BH][grid_h][grid_w][d]; 3: text prefix of q as [BH][n_text][d];
+// 4, 5: k, v as the token sequence [BH][N][d].
+int build_maps(const clear_plan &p, const void *q, const void *k, const void *v)
+{
+    const Shape &s = p.shape;
+    const uint64_t d = (uint64_t)s.head_dim, gw = (uint64_t)s.grid_w, gh = (uint64_t)s.grid_h, T = (uint64_t)s.n_text;
+    const uint64_t N = T + gw * gh, BH = (uint64_t)s.B * s.H;
+    const uint64_t row_b = d * 2;
+    CUtensorMap *tm = reinterpret_cast<CUtensorMap *>(p.tm_storage);
+    const void *ptrs[3] = {q, k, v};
+    const uint64_t dims4[4] = {d, gw, gh, BH};
+    const uint64_t str4[3] = {row_b, gw * row_b, N * row_b};
+    const uint32_t box4[4] = {64, (uint32_t)kTileW, (uint32_t)kTileH, 1};
+    for (int t = 0; t < 3; ++t) {
+        const char *base = static_cast<const char *>(ptrs[t]) + T * row_b;
+        if (!encode(&tm[t], base, 4, dims4, str4, box4)) return CLEAR_ERR_CUDA;
+    }
+    const uint64_t dims3[3] = {d, N, BH};
+    const uint64_t dims3t[3] = {d, T > 0 ? T : 1, BH};
+    const uint64_t str3[2] = {row_b, N * row_b};
+    const uint32_t box3[3] = {64, (uint32_t)kTileTokens, 1};
+    if (!encode(&tm[3], q, 3, dims3t, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode(&tm[4], k, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode(&tm[5], v, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
+    for (int t = 0; t < 3; ++t) p.tm_ptrs[t] = ptrs[t];
+    p.tm_ptrs[3] = nullptr;
+    p.tm_valid = true;
+    return CLEAR_OK;
+}
+
+struct DeviceInfo {
+    bool known = false;
+    int n_sm = 0;
+    bool configured[2] = {false, false};
+};
+DeviceInfo g_dev[64];
+std::mutex g_dev_mutex;
+
+template <int D>
+int launch_variant(const clear_plan &p, const CUtensorMap *tm, const WsParams &prm, cudaStream_t stream)
+{
+    constexpr size_t kSmem = (size_t)(2 + kRing) * (D / 64) * 16384 + sizeof(Ctrl);
+    static_assert(kSmem <= 232448, "shared memory of one block");
+    int n_sm = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_dev_mutex);
+        if (p.device < 0 || p.device >= 64) return CLEAR_ERR_UNSUPPORTED;
+        DeviceInfo &di = g_dev[p.device];
+        if (!di.known) {
+            CLEAR_CUDA_TRY(cudaDeviceGetAttribute(&di.n_sm, cudaDevAttrMultiProcessorCount, p.device));
+            di.known = true;
+        }
+        if (!di.configured[D == 128]) {
+            CLEAR_CUDA_TRY(cudaFuncSetAttribute(clear_ws_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem));
+            di.configured[D == 128] = true;
+        }
+        n_sm = di.n_sm;
+    }
+    const long long total = (long long)prm.n_items * prm.n_bh;
+    const unsigned grid = (unsigned)std::min<long long>(n_sm, total);
+    clear_ws_kernel<D><<<grid, kWsThreads, kSmem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], prm);
+    CLEAR_CUDA_TRY(cudaGetLastError());
+    return launch_text_combine(p, prm.out, stream);
+}
+
+}  // namespace
+
+int launch_ws(const clear_plan &p, const void *q, const void *k, const void *v, void *out, float scale,
+              cudaStream_t stream)
+{
+    if (!(scale > 0.f)) return CLEAR_ERR_UNSUPPORTED;
+    const long long total = (long long)p.sch.pair_items.size() * p.shape.B * p.shape.H;
+    if (total <= 0 || total >= (1ll << 30)) return CLEAR_ERR_UNSUPPORTED;
+    CUtensorMap tm[6];
+    {
+        std::lock_guard<std::mutex> lock(p.tm_mutex);
+        if (!(p.tm_valid && p.tm_ptrs[0] == q && p.tm_ptrs[1] == k && p.tm_ptrs[2] == v)) {
+            int rc = build_maps(p, q, k, v);
+            if (rc != CLEAR_OK) {
+                p.tm_valid = false;
+                return rc;
+            }
+        }
+        std::memcpy(tm, p.tm_storage, sizeof(tm));
+    }
+    WsParams prm;
+    prm.items = p.d_pair_items;
+    prm.steps = p.d_pair_steps;
+    prm.half_width = p.d_half_width;
+    prm.n_half_width = (int)p.sch.half_width.size();
+    prm.grid_h = p.shape.grid_h;
+    prm.grid_w = p.shape.grid_w;
+    prm.n_text = p.shape.n_text;
+    prm.n_tokens = (long long)p.shape.n_text + (long long)p.shape.grid_h * p.shape.grid_w;
+    prm.n_items = (int)p.sch.pair_items.size();
+    prm.n_text_items = p.sch.n_text_pair_items;
+    prm.n_bh = p.shape.B * p.shape.H;
+    prm.scale_log2 = scale * 1.4426950408889634f;
+    prm.partial_o = p.d_partial_o;
+    prm.partial_ml = p.d_partial_ml;
+    prm.n_partial_slots = p.sch.n_partial_slots;
+    prm.out = static_cast<__nv_bfloat16 *>(out);
+    prm.status = p.d_status;
+    if (p.shape.head_dim == 128) return launch_variant<128>(p, tm, prm, stream);
+    if (p.shape.head_dim == 64) return launch_variant<64>(p, tm, prm, stream);
+    return CLEAR_ERR_UNSUPPORTED;
+}
+
+}  // namespace clear

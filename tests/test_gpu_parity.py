@@ -116,19 +116,42 @@ TC_SMALL = [
 ]
 
 
+TC_KERNELS = [clear.KERNEL_TCGEN05_WS, clear.KERNEL_TCGEN05]
+TC_IDS = ["ws", "tile"]
+
+
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_IDS)
 @pytest.mark.parametrize("gh,gw,T,r,d", TC_SMALL)
-def test_tc_kernel_small_shapes(gh, gw, T, r, d):
+def test_tc_kernel_small_shapes(gh, gw, T, r, d, kernel):
     q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=gh * 1000 + gw * 10 + T)
     scale = 1 / math.sqrt(d)
     want = oracle.attn(q, k, v, gh, gw, T, r, scale)
-    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05)
+    got = run_plan(q, k, v, gh, gw, T, r, scale, kernel)
     assert_close_bf16(got, want, f"tc {gh}x{gw}+{T} r={r} d={d}")
 
 
-def test_tc_kernel_split_text_rows_small():
+def test_ws_kernel_many_heads_keep_the_queue_busy():
+    """More (batch, head) pairs than SMs' worth of items: every block takes many items from the queue."""
+    gh, gw, T, r, d = 48, 64, 300, 7.0, 128
+    q, k, v = workloads.make_custom(2, 12, gh, gw, T, d, seed=4242)
+    scale = 1 / math.sqrt(d)
+    rng = np.random.default_rng(5)
+    rows = np.array([(b, h, int(i)) for b in range(2) for h in range(12)
+                     for i in list(rng.integers(0, T + gh * gw, 24)) + [0, T - 1, T, T + gh * gw - 1]], dtype=np.int64)
+    want = oracle.attn_rows(q, k, v, gh, gw, T, r, scale, rows)
+    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05_WS)
+    assert torch.isfinite(got.float()).all(), "some output element was never written"
+    assert_close_bf16(got[rows[:, 0], rows[:, 1], rows[:, 2]], want, "many heads")
+    # and the two tensor-core kernels agree everywhere (same arithmetic, different schedule)
+    other = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05)
+    assert float((got.float() - other.float()).abs().max()) <= 2e-2
+
+
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_IDS)
+def test_tc_kernel_split_text_rows_small(kernel):
     """N large enough that the text-query rows are split over key ranges and merged."""
     gh, gw, T, r, d = 96, 96, 200, 6.0, 128
-    plan = clear.Plan(1, 1, gh, gw, T, d, r, host_only=True)
+    plan = clear.Plan(1, 1, gh, gw, T, d, r, kernel=kernel, host_only=True)
     assert plan.info().n_text_splits > 1
     q, k, v = workloads.make_custom(1, 1, gh, gw, T, d, seed=77)
     scale = 1 / math.sqrt(d)
@@ -136,24 +159,26 @@ def test_tc_kernel_split_text_rows_small():
     rows = np.array([(0, 0, i) for i in list(range(0, T, 7)) + [T - 1] +
                      [T + int(p) for p in rng.integers(0, gh * gw, 200)]], dtype=np.int64)
     want = oracle.attn_rows(q, k, v, gh, gw, T, r, scale, rows)
-    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05)
+    got = run_plan(q, k, v, gh, gw, T, r, scale, kernel)
     assert_close_bf16(got[rows[:, 0], rows[:, 1], rows[:, 2]], want, "split text rows")
 
 
-def test_tc_kernel_large_logits_exercise_the_rescale_path():
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_IDS)
+def test_tc_kernel_large_logits_exercise_the_rescale_path(kernel):
     """Un-normalised Q, K: row maxima jump by far more than the lazy-rescale threshold."""
     gh, gw, T, r, d = 24, 32, 64, 6.0, 128
     q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, qk_norm=False, seed=9)
     scale = 1.0
     want = oracle.attn(q, k, v, gh, gw, T, r, scale)
-    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05)
+    got = run_plan(q, k, v, gh, gw, T, r, scale, kernel)
     assert_close_bf16(got, want, "large logits")
 
 
 # ----------------------------------------------------------------------------------------------
 # mask exactness through bf16: uniform softmax reads membership and counts
 # ----------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("kernel", [clear.KERNEL_TCGEN05, clear.KERNEL_SIMT])
+@pytest.mark.parametrize("kernel", [clear.KERNEL_TCGEN05_WS, clear.KERNEL_TCGEN05, clear.KERNEL_SIMT],
+                         ids=["ws", "tile", "simt"])
 @pytest.mark.parametrize("gh,gw,T,r", [(24, 40, 5, 8.0), (19, 23, 0, 4.0), (16, 48, 130, 3.0)])
 def test_zero_queries_read_back_the_mask(kernel, gh, gw, T, r):
     """Q = 0: out_i = mean of V over the allowed set.  V column c is one-hot on a planted key, so
@@ -207,7 +232,7 @@ def test_planted_key_at_the_radius_threshold():
     want = oracle.attn_rows(q, k, v, gh, gw, T, r, 1.0, rows)
     assert np.abs(want[0] - v[0, 0, inside].double().numpy()).max() < 1e-2   # the oracle picks `inside`
     assert np.abs(want[1] - v[0, 0, wrap].double().numpy()).max() > 0.5      # and never sees `wrap`
-    for kernel in (clear.KERNEL_TCGEN05, clear.KERNEL_SIMT):
+    for kernel in (clear.KERNEL_TCGEN05_WS, clear.KERNEL_TCGEN05, clear.KERNEL_SIMT):
         got = run_plan(q, k, v, gh, gw, T, r, 1.0, kernel)[0, 0, [qa, qb]].double().numpy()
         assert np.abs(got - want).max() < 2e-2
 
@@ -268,7 +293,8 @@ def test_rows_stay_normalised_at_full_size():
 # ----------------------------------------------------------------------------------------------
 # robustness of the boundary
 # ----------------------------------------------------------------------------------------------
-def test_guard_bands_repeat_calls_and_streams():
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_IDS)
+def test_guard_bands_repeat_calls_and_streams(kernel):
     gh, gw, T, r, d = 24, 40, 130, 8.0, 128
     q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=21)
     scale = 1 / math.sqrt(d)
@@ -277,7 +303,7 @@ def test_guard_bands_repeat_calls_and_streams():
     buf = torch.full((n + 2 * guard,), -7.0, dtype=torch.bfloat16, device=dev())
     out = buf[guard: guard + n].view(q.shape)
     qd, kd, vd = (t.to(dev()) for t in (q, k, v))
-    plan = clear.Plan(1, 2, gh, gw, T, d, r, kernel=clear.KERNEL_TCGEN05)
+    plan = clear.Plan(1, 2, gh, gw, T, d, r, kernel=kernel)
     plan.forward(qd, kd, vd, out, scale)
     plan.check()
     first = out.clone()
@@ -308,10 +334,11 @@ def test_device_side_argument_errors():
     p = x.data_ptr()
     assert lib.clear_attn_fwd(p, p, p, p + 2, 1, 1, 16, 16, 16, 64, 4.0, 0.125, None) == clear.ERR_MISALIGNED
     assert lib.clear_attn_fwd(p, p, p, None, 1, 1, 16, 16, 16, 64, 4.0, 0.125, None) == clear.ERR_INVALID_ARG
-    plan = clear.Plan(1, 1, 16, 16, 16, 64, 4.0, kernel=clear.KERNEL_TCGEN05)
-    out = torch.empty_like(x)
-    assert lib.clear_attn_fwd_planned(plan.handle, p, p, p, out.data_ptr(), -1.0, None) == clear.ERR_UNSUPPORTED
-    plan.destroy()
+    for kernel in TC_KERNELS:
+        plan = clear.Plan(1, 1, 16, 16, 16, 64, 4.0, kernel=kernel)
+        out = torch.empty_like(x)
+        assert lib.clear_attn_fwd_planned(plan.handle, p, p, p, out.data_ptr(), -1.0, None) == clear.ERR_UNSUPPORTED
+        plan.destroy()
 
 
 def test_host_tensor_entry_point():

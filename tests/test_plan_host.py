@@ -50,6 +50,9 @@ def test_status_strings():
     (dict(head_dim=512), clear.ERR_UNSUPPORTED), (dict(head_dim=20), clear.ERR_UNSUPPORTED),
     (dict(head_dim=96, kernel=clear.KERNEL_TCGEN05), clear.ERR_UNSUPPORTED),
     (dict(dtype=clear.F32, kernel=clear.KERNEL_TCGEN05), clear.ERR_UNSUPPORTED),
+    (dict(head_dim=96, kernel=clear.KERNEL_TCGEN05_WS), clear.ERR_UNSUPPORTED),
+    (dict(dtype=clear.F32, kernel=clear.KERNEL_TCGEN05_WS), clear.ERR_UNSUPPORTED),
+    (dict(kernel=4), clear.ERR_INVALID_ARG),
 ])
 def test_plan_rejects_bad_shapes(kwargs, status):
     base = dict(B=1, H=2, grid_h=16, grid_w=16, n_text=16, head_dim=64, radius=4.0, dtype=clear.BF16,
@@ -76,8 +79,10 @@ def test_host_plan_cannot_run_and_null_arguments_are_rejected():
 
 
 def test_kernel_selection():
-    assert clear.Plan(1, 1, 16, 16, 16, 128, 4.0, host_only=True).info().kernel == clear.KERNEL_TCGEN05
-    assert clear.Plan(1, 1, 16, 16, 16, 64, 4.0, host_only=True).info().kernel == clear.KERNEL_TCGEN05
+    assert clear.Plan(1, 1, 16, 16, 16, 128, 4.0, host_only=True).info().kernel == clear.KERNEL_TCGEN05_WS
+    assert clear.Plan(1, 1, 16, 16, 16, 64, 4.0, host_only=True).info().kernel == clear.KERNEL_TCGEN05_WS
+    assert clear.Plan(1, 1, 16, 16, 16, 64, 4.0, kernel=clear.KERNEL_TCGEN05,
+                      host_only=True).info().kernel == clear.KERNEL_TCGEN05
     assert clear.Plan(1, 1, 16, 16, 16, 96, 4.0, host_only=True).info().kernel == clear.KERNEL_SIMT
     assert clear.Plan(1, 1, 16, 16, 16, 64, 4.0, dtype=clear.F32, host_only=True).info().kernel == clear.KERNEL_SIMT
 
@@ -89,7 +94,7 @@ SHAPES = [(16, 16, 16, 4.0), (13, 19, 7, 4.0), (24, 40, 130, 8.0), (9, 33, 0, 5.
 @pytest.mark.parametrize("gh,gw,T,r", SHAPES)
 def test_geometry_matches_the_oracle_mask(gh, gw, T, r):
     total, counts = oracle.mask_counts(gh, gw, T, r)
-    for kernel in (clear.KERNEL_SIMT, clear.KERNEL_TCGEN05):
+    for kernel in (clear.KERNEL_SIMT, clear.KERNEL_TCGEN05, clear.KERNEL_TCGEN05_WS):
         p = clear.Plan(2, 3, gh, gw, T, 64, r, kernel=kernel, host_only=True)
         info = p.info()
         assert info.sum_mask == total
@@ -183,8 +188,129 @@ def test_tile_schedule_covers_each_allowed_pair_exactly_once(gh, gw, T, r):
         assert info.workspace_bytes == len(slots) * 128 * (128 + 2) * 4
 
 
-def test_text_rows_are_split_for_long_sequences():
+def key_tokens(x, y, linear, n_valid, gh, gw, T, th, tw):
+    """Token indices a key tile holds (existing keys only), and whether all 128 exist."""
+    if linear:
+        return np.arange(x, x + n_valid), n_valid == 128
+    ys, xs = np.meshgrid(np.arange(y, y + th), np.arange(x, x + tw), indexing="ij")
+    ok = (ys >= 0) & (ys < gh) & (xs >= 0) & (xs < gw)
+    return (T + ys * gw + xs)[ok], bool(ok.all())
+
+
+@pytest.mark.parametrize("gh,gw,T,r", SHAPES + [(40, 40, 300, 9.0), (17, 16, 129, 4.0)])
+def test_pair_schedule_covers_each_allowed_pair_exactly_once(gh, gw, T, r):
+    p = clear.Plan(1, 1, gh, gw, T, 128, r, kernel=clear.KERNEL_TCGEN05_WS, host_only=True)
+    info = p.info()
+    items, steps = p.pair_tables()
+    N = T + gh * gw
+    th, tw = info.tile_h, info.tile_w
+    assert th * tw == 128 and info.n_work_items == len(items)
+    n_text_items = sum(1 for it in items if it.kind == 1)
+    assert all(it.kind == 1 for it in items[:n_text_items]) and all(it.kind == 0 for it in items[n_text_items:])
+    img_counts = [it.step_count for it in items[n_text_items:]]
+    assert img_counts == sorted(img_counts, reverse=True)
+    assert info.max_item_tiles == max(it.step_count for it in items)
+
+    executed = 0
+    seen_queries = np.zeros(N, dtype=np.int64)
+    text_cover = {}
+    slots = set()
+    for it in items:
+        assert it.step_count >= 1 and it.n_sides in (1, 2)
+        sts = steps[it.step_begin: it.step_begin + it.step_count]
+        # ring bookkeeping: K and V of each distinct key tile of a step take one stage each
+        loads = 0
+        for st in sts:
+            assert st.load_base == loads
+            use0, use1 = bool(st.flags & clear.STEP_USE0), bool(st.flags & clear.STEP_USE1)
+            shared = bool(st.flags & clear.STEP_SHARED)
+            assert use0 or use1
+            if shared:
+                assert use0 and use1 and (st.x0, st.y0) == (st.x1, st.y1)
+            if it.n_sides == 1:
+                assert not use1
+            if use0 and use1 and not shared and not (st.flags & clear.STEP_LINEAR):
+                assert (st.x0, st.y0) != (st.x1, st.y1)
+            loads += 2 * (int(use0) + int(use1 and not shared))
+            executed += (int(use0) + int(use1)) * 128 * 128
+        assert it.n_loads == loads
+        for side in range(it.n_sides):
+            use_bit = clear.STEP_USE1 if side else clear.STEP_USE0
+            mask_bit = clear.STEP_MASKED1 if side else clear.STEP_MASKED0
+            mine = [st for st in sts if st.flags & use_bit]
+            assert mine, "a query tile with no key tile"
+            tiles = [((st.x1, st.y1, st.n_valid1) if side else (st.x0, st.y0, st.n_valid0)) +
+                     (bool(st.flags & clear.STEP_LINEAR), bool(st.flags & mask_bit)) for st in mine]
+            slot = it.partial_slot1 if side else it.partial_slot0
+            n_rows = it.n_rows1 if side else it.n_rows0
+            if it.kind == 1:
+                q0 = it.qx + 128 * side
+                assert q0 % 128 == 0 and n_rows == min(128, T - q0) and n_rows > 0
+                toks = []
+                for (x, y, nv, linear, masked) in tiles:
+                    assert linear and nv == min(128, N - x) and masked == (nv < 128)
+                    toks += list(range(x, x + nv))
+                assert toks == list(range(toks[0], toks[-1] + 1))
+                text_cover.setdefault(q0, []).extend(toks)
+                if info.n_text_splits > 1:
+                    assert slot >= 0 and slot not in slots and slot // info.n_text_splits == q0 // 128
+                    slots.add(slot)
+                else:
+                    assert slot == -1
+                continue
+            qy = it.qy1 if side else it.qy0
+            assert slot == -1 and it.qx % tw == 0 and qy % th == 0
+            if side:
+                assert it.qy1 == it.qy0 + th
+            qs = [(y, x) for y in range(qy, min(qy + th, gh)) for x in range(it.qx, min(it.qx + tw, gw))]
+            assert n_rows == len(qs) and n_rows > 0
+            cover = np.zeros(N, dtype=np.int64)
+            unmasked = np.zeros(N, dtype=bool)
+            rows = {q: oracle.mask_row(T + q[0] * gw + q[1], gh, gw, T, r).astype(bool) for q in qs}
+            for (x, y, nv, linear, masked) in tiles:
+                idx, whole = key_tokens(x, y, linear, nv, gh, gw, T, th, tw)
+                if linear:
+                    assert x + nv <= T and masked == (nv < 128)
+                else:
+                    # no useless tile: it holds at least one allowed pair
+                    assert any(rows[q][idx].any() for q in qs)
+                    if not masked:
+                        assert whole
+                        unmasked[idx] = True
+                cover[idx] += 1
+            assert cover.max() <= 1
+            for q in qs:
+                seen_queries[T + q[0] * gw + q[1]] += 1
+                assert not (rows[q] & (cover == 0)).any(), "an allowed key is in no tile of the query tile"
+                assert rows[q][unmasked].all(), "a tile flagged mask-free holds a disallowed pair"
+    assert info.executed_pairs == executed
+    assert np.all(seen_queries[T:] == 1)
+    for q0 in range(0, T, 128):
+        assert sorted(text_cover[q0]) == list(range(N))
+    if info.n_text_splits > 1:
+        assert len(slots) == math.ceil(T / 128) * info.n_text_splits
+        assert info.workspace_bytes == len(slots) * 128 * (128 + 2) * 4
+
+
+def test_pair_schedule_at_the_8k_workload():
     p = clear.Plan(1, 24, 512, 512, 512, 128, 16.0, host_only=True)
+    info = p.info()
+    assert info.kernel == clear.KERNEL_TCGEN05_WS
+    assert info.sum_mask == 471125568
+    items, steps = p.pair_tables()
+    interior = [it for it in items if it.kind == 0 and it.step_count == 19]
+    assert len(interior) > 800                           # 4 text + 3 one-sided pairs + 12 shared key patches
+    it = interior[0]
+    sts = steps[it.step_begin: it.step_begin + it.step_count]
+    assert sum(1 for st in sts if st.flags & clear.STEP_SHARED) == 16 and it.n_loads == 2 * 22
+    # every query tile still executes 19 key tiles: the same geometric efficiency as one tile per block
+    one = clear.Plan(1, 24, 512, 512, 512, 128, 16.0, kernel=clear.KERNEL_TCGEN05, host_only=True).info()
+    assert info.executed_pairs == one.executed_pairs
+    assert max(it.step_count for it in items) <= 64
+
+
+def test_text_rows_are_split_for_long_sequences():
+    p = clear.Plan(1, 24, 512, 512, 512, 128, 16.0, kernel=clear.KERNEL_TCGEN05, host_only=True)
     info = p.info()
     assert info.kernel == clear.KERNEL_TCGEN05
     assert info.sum_mask == 471125568                   # matches the 5.79 TFLOPS cell of the paper
