@@ -37,8 +37,9 @@ constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when
 constexpr int kSchedDepth = 2;
 // arrivals that free a queue slot: the MMA thread and one lane of each of the 12 softmax / epilogue warps
 constexpr uint32_t kSchedReaders = 13;
-// registers per thread of each role (warpgroups of 128 threads: 48 + 2 * 192 + 80 = 512)
-constexpr uint32_t kRegsControl = 48, kRegsSoftmax = 192, kRegsEpilogue = 80;
+// registers per thread of each role (warpgroups of 128 threads: 72 + 2 * 184 + 72 = 512)
+constexpr uint32_t kRegsControl = 72, kRegsSoftmax = 184, kRegsEpilogue = 72;
+constexpr int kHalfWidthSmem = 128;  // entries of the half-width table kept in shared memory
 
 struct WsParams {
     const clear_pair_item_t *items;
@@ -62,11 +63,14 @@ struct Ctrl {
     uint64_t s_full[2], p_ready[2], o_full[2], o_empty[2], stats_full[2], stats_empty[2];
     uint64_t sched_full[kSchedDepth], sched_empty[kSchedDepth];
     uint64_t drain;
-    int32_t sched_item[kSchedDepth];
+    int32_t sched_item[kSchedDepth];            // queue position, >= total: no more work
+    int32_t sched_bh[kSchedDepth];
+    clear_pair_item_t sched_rec[kSchedDepth];   // the item's record, read once from global memory
     uint32_t tmem_base;
     int abort_flag;
     int skip;
     float2 stats[2][128];  // per query row: running maximum (log2 units) and row sum
+    int32_t half_width[kHalfWidthSmem];
 };
 
 // Bounded wait on an mbarrier phase.  Returns false once the block has given up.
@@ -130,6 +134,21 @@ __device__ __forceinline__ clear_pair_item_t load_item(const clear_pair_item_t *
     it.qy1 = b.x; it.n_rows0 = b.y; it.n_rows1 = b.z; it.step_begin = b.w;
     it.step_count = c.x; it.n_loads = c.y; it.partial_slot0 = c.z; it.partial_slot1 = c.w;
     return it;
+}
+// The part of a step record one query tile of the pair needs.
+struct SideStep {
+    int x, y, flags, n_valid;
+};
+__device__ __forceinline__ SideStep load_side_step(const clear_pair_step_t *p, int side)
+{
+    const int4 a = __ldg(reinterpret_cast<const int4 *>(p));
+    const int4 b = __ldg(reinterpret_cast<const int4 *>(p) + 1);
+    SideStep s;
+    s.x = side ? a.z : a.x;
+    s.y = side ? a.w : a.y;
+    s.flags = b.x;
+    s.n_valid = side ? b.z : b.y;
+    return s;
 }
 static_assert(sizeof(clear_pair_step_t) == 32 && sizeof(clear_pair_item_t) == 48, "table records are read as int4");
 
@@ -222,6 +241,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         ptx::mbar_init(ptx::smem_u32(&ctrl->drain), 1);
         ptx::fence_mbar_init();
     }
+    for (int i = tid; i < prm.n_half_width && i < kHalfWidthSmem; i += kWsThreads) ctrl->half_width[i] = prm.half_width[i];
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), kTmemCols);
         ptx::tmem_relinquish();
@@ -241,11 +261,17 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
                 if (!wait_bar(ptx::smem_u32(&ctrl->sched_empty[slot]), (use & 1u) ^ 1u, abort_flag, prm.status, 1)) break;
                 const int g = atomicAdd(prm.status + 1, 1);
+                ItemRef ref{0, 0};
+                clear_pair_item_t item{};
+                if (g < total_items) {
+                    ref = decode_item(prm, g);
+                    item = load_item(prm.items + ref.item);
+                    ctrl->sched_rec[slot] = item;
+                    ctrl->sched_bh[slot] = ref.bh;
+                }
                 ctrl->sched_item[slot] = g;
                 ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_full[slot]));
                 if (g >= total_items) break;
-                const ItemRef ref = decode_item(prm, g);
-                const clear_pair_item_t item = load_item(prm.items + ref.item);
                 bool ok = true;
                 for (int t = 0; t < item.n_sides && ok; ++t) {
                     const uint32_t bar = ptx::smem_u32(&ctrl->q_full[t]);
@@ -263,8 +289,11 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     ++n_q[t];
                 }
                 const clear_pair_step_t *steps = prm.steps + item.step_begin;
+                clear_pair_step_t st_next = load_step(steps);
                 for (int s = 0; s < item.step_count && ok; ++s) {
-                    const clear_pair_step_t st = load_step(steps + s);
+                    // the next record is fetched one step ahead, so its latency is off the critical path
+                    const clear_pair_step_t st = st_next;
+                    if (s + 1 < item.step_count) st_next = load_step(steps + s + 1);
                     const bool has_a = (st.flags & CLEAR_STEP_USE0) != 0;
                     const bool has_b = (st.flags & CLEAR_STEP_USE1) && !(st.flags & CLEAR_STEP_SHARED);
                     const bool linear = (st.flags & CLEAR_STEP_LINEAR) != 0;
@@ -317,10 +346,9 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
                 if (!wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 5)) break;
                 const int g = ctrl->sched_item[slot];
+                const clear_pair_item_t item = ctrl->sched_rec[slot];
                 ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
                 if (g >= total_items) break;
-                const ItemRef ref = decode_item(prm, g);
-                const clear_pair_item_t item = load_item(prm.items + ref.item);
                 const clear_pair_step_t *steps = prm.steps + item.step_begin;
                 const int n = item.step_count;
                 for (int t = 0; t < item.n_sides && ok; ++t)
@@ -408,6 +436,8 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
         const float c = prm.scale_log2;
+        // the table of Eq. 3's half widths: shared memory when it fits, else global memory
+        const int32_t *half_width = prm.n_half_width <= kHalfWidthSmem ? ctrl->half_width : prm.half_width;
         const uint32_t b_s = ptx::smem_u32(&ctrl->s_full[t]), b_p = ptx::smem_u32(&ctrl->p_ready[t]);
         uint32_t n_s = 0, n_items_seen = 0;
         bool alive = true;
@@ -416,11 +446,10 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 9)))
                 break;
             const int g = ctrl->sched_item[slot];
+            const clear_pair_item_t item = ctrl->sched_rec[slot];
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
             if (g >= total_items) break;
-            const ItemRef ref = decode_item(prm, g);
-            const clear_pair_item_t item = load_item(prm.items + ref.item);
             if (t >= item.n_sides) continue;
             const clear_pair_step_t *steps = prm.steps + item.step_begin;
             const bool is_text = item.kind == 1;
@@ -436,19 +465,20 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
 
+            SideStep st_next = load_side_step(steps, t);
             for (int s = 0; s < item.step_count; ++s) {
-                const clear_pair_step_t st = load_step(steps + s);
+                // the next record is fetched one step ahead, so its latency is off the critical path
+                const SideStep st = st_next;
+                if (s + 1 < item.step_count) st_next = load_side_step(steps + s + 1, t);
                 if (!step_uses(st.flags, t)) continue;
                 const bool masked = (st.flags & (t ? CLEAR_STEP_MASKED1 : CLEAR_STEP_MASKED0)) != 0;
-                const int k_x = t ? st.x1 : st.x0, k_y = t ? st.y1 : st.y0;
                 // ---- mask bits of this row for the tile (bit j = key j allowed) -----------------------
                 uint32_t mw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
                 if (masked) {
                     if (st.flags & CLEAR_STEP_LINEAR) {
-                        const int n_valid = t ? st.n_valid1 : st.n_valid0;
 #pragma unroll
                         for (int w = 0; w < 4; ++w) {
-                            const int nv = min(max(n_valid - 32 * w, 0), 32);
+                            const int nv = min(max(st.n_valid - 32 * w, 0), 32);
                             mw[w] = nv == 32 ? 0xffffffffu : ((1u << nv) - 1u);
                         }
                     } else {
@@ -456,14 +486,14 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         for (int w = 0; w < 4; ++w) mw[w] = 0u;
 #pragma unroll
                         for (int rr = 0; rr < 8; ++rr) {
-                            const int ky = k_y + rr;
+                            const int ky = st.y + rr;
                             const int ady = abs(ky - q_y);
                             uint32_t bits = 0u;
                             if (q_valid && ky >= 0 && ky < prm.grid_h && ady < prm.n_half_width) {
-                                const int hw = __ldg(prm.half_width + ady);
-                                const int lo = max(max(q_x - hw, 0), k_x);
-                                const int hi = min(min(q_x + hw, prm.grid_w - 1), k_x + 15);
-                                if (lo <= hi) bits = ((1u << (hi - lo + 1)) - 1u) << (lo - k_x);
+                                const int hw = half_width[ady];
+                                const int lo = max(max(q_x - hw, 0), st.x);
+                                const int hi = min(min(q_x + hw, prm.grid_w - 1), st.x + 15);
+                                if (lo <= hi) bits = ((1u << (hi - lo + 1)) - 1u) << (lo - st.x);
                             }
                             mw[rr >> 1] |= bits << (16 * (rr & 1));
                         }
@@ -482,22 +512,27 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 for (int w = 0; w < 4; ++w) ptx::tmem_ld32(tmem_S + lane_off + 32 * w, sv[w]);
                 ptx::tmem_wait_ld();
 
-                float mx = -INFINITY;
+                // row maximum over the allowed keys, four independent chains of three-input maxima
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 if (masked) {
 #pragma unroll
                     for (int w = 0; w < 4; ++w)
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const float val = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
-                            sv[w][j] = __float_as_uint(val);
-                            mx = fmaxf(mx, val);
+                        for (int j = 0; j < 32; j += 2) {
+                            const float v0 = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
+                            const float v1 = ((mw[w] >> (j + 1)) & 1u) ? __uint_as_float(sv[w][j + 1]) : -INFINITY;
+                            sv[w][j] = __float_as_uint(v0);
+                            sv[w][j + 1] = __float_as_uint(v1);
+                            mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], v0, v1);
                         }
                 } else {
 #pragma unroll
                     for (int w = 0; w < 4; ++w)
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(sv[w][j]));
+                        for (int j = 0; j < 32; j += 2)
+                            mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], __uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1]));
                 }
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
 
                 // ---- running maximum; O is rescaled only when it grew by more than the threshold -----
                 const float m_new = fmaxf(m_used, mx);
@@ -528,17 +563,28 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 const float mc = (m_used == -INFINITY) ? 0.f : m_used * c;
 
                 // ---- P = exp2(S * c - m * c), row sum, bf16 pairs over the first 64 columns of S -----
+                // (two-wide fp32 FMA and ADD; four independent partial sums)
+                const uint64_t c2 = ptx::pack2(c, c), nmc2 = ptx::pack2(-mc, -mc);
+                uint64_t lsum[2] = {0ull, 0ull};
 #pragma unroll
                 for (int w = 0; w < 4; ++w) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
-                        const float p0 = ptx::ex2(fmaf(__uint_as_float(sv[w][j]), c, -mc));
-                        const float p1 = ptx::ex2(fmaf(__uint_as_float(sv[w][j + 1]), c, -mc));
-                        l += p0 + p1;
+                        const uint64_t x2 = ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
+                        float x0, x1;
+                        ptx::unpack2(x2, x0, x1);
+                        const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
+                        lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
                         pk[j >> 1] = ptx::pack_bf16(p0, p1);
                     }
                     ptx::tmem_st16(tmem_S + lane_off + 16 * w, pk);
+                }
+                {
+                    float a0, a1, a2, a3;
+                    ptx::unpack2(lsum[0], a0, a1);
+                    ptx::unpack2(lsum[1], a2, a3);
+                    l += (a0 + a1) + (a2 + a3);
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before();
@@ -566,11 +612,12 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 12)))
                 break;
             const int g = ctrl->sched_item[slot];
+            const clear_pair_item_t item = ctrl->sched_rec[slot];
+            ItemRef ref;
+            ref.bh = ctrl->sched_bh[slot];
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
             if (g >= total_items) break;
-            const ItemRef ref = decode_item(prm, g);
-            const clear_pair_item_t item = load_item(prm.items + ref.item);
             for (int t = 0; t < item.n_sides; ++t) {
                 const uint32_t ph = n_seen[t] & 1u;
                 if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->stats_full[t]), ph, abort_flag, prm.status, 13))) {
