@@ -247,6 +247,12 @@ const char *clear_status_string(int status);
 /* cudaError_t value of the most recent CUDA failure seen by the calling thread (0 if none). */
 int clear_last_cuda_error(void);
 
+/* Diagnostic detail of the most recent CLEAR_ERR_DEVICE_TIMEOUT returned to the calling thread by
+ * clear_plan_check or clear_attn_fwd_host: the non-zero word the kernel left in the plan's status
+ * slot, which names the wait that expired (a kernel-internal code, stable only within one build).
+ * 0 if there was none. */
+int clear_last_device_status(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,13 +26,15 @@ EXPORTS = [
     "clear_plan_tables", "clear_attn_fwd_planned", "clear_attn_fwd_host", "clear_plan_info",
     "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
     "clear_last_cuda_error", "clear_attn_fwd_static", "clear_plan_pair_tables",
+    "clear_last_device_status",
 ]
 
 
 class ClearError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
-        super().__init__(f"{what}: {status_string(status)} (status {status}, cuda error {last_cuda_error()})")
+        detail = f", device status {last_device_status()}" if status == ERR_DEVICE_TIMEOUT else ""
+        super().__init__(f"{what}: {status_string(status)} (status {status}, cuda error {last_cuda_error()}{detail})")
 
 
 class PlanInfo(ctypes.Structure):
@@ -107,6 +109,7 @@ def load() -> ctypes.CDLL:
         lib.clear_status_string.argtypes = [i32]
         lib.clear_status_string.restype = ctypes.c_char_p
         lib.clear_last_cuda_error.argtypes = []
+        lib.clear_last_device_status.argtypes = []
         for name in EXPORTS:
             if name != "clear_status_string":
                 getattr(lib, name).restype = i32
@@ -120,6 +123,11 @@ def status_string(status: int) -> str:
 
 def last_cuda_error() -> int:
     return int(load().clear_last_cuda_error())
+
+
+def last_device_status() -> int:
+    """Kernel-internal code of the wait that expired in the last DEVICE_TIMEOUT seen by this thread."""
+    return int(load().clear_last_device_status())
 
 
 def _check(status: int, what: str) -> None:

@@ -11,6 +11,7 @@
 namespace clear {
 
 static thread_local int g_last_cuda_error = 0;
+static thread_local int g_last_device_status = 0;
 void note_cuda_error(int err) { g_last_cuda_error = err; }
 
 namespace {
@@ -329,6 +330,7 @@ int clear_plan_check(clear_plan_t *plan, void *stream)
     CLEAR_CUDA_TRY(cudaMemcpyAsync(&status, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost, cs));
     CLEAR_CUDA_TRY(cudaStreamSynchronize(cs));
     if (status != 0) {
+        g_last_device_status = status;
         // a block that gave up may have left the work queue of the persistent kernel mid-way
         CLEAR_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, kStatusWords * sizeof(int), cs));
         CLEAR_CUDA_TRY(cudaStreamSynchronize(cs));
@@ -386,5 +388,7 @@ const char *clear_status_string(int status)
 }
 
 int clear_last_cuda_error(void) { return g_last_cuda_error; }
+
+int clear_last_device_status(void) { return g_last_device_status; }
 
 }  // extern "C"

@@ -7,8 +7,8 @@
 //
 // Roles (512 threads):
 //   warp 0        : takes items from the queue and issues every TMA load (Q tiles, K/V ring);
-//   warp 1        : issues every tcgen05.mma: S_t = Q_t K^T, O_t += P_t V, t = 0, 1, interleaved so
-//                   that the softmax of one query tile runs under the MMAs of the other;
+//   warps 1, 2    : one thread each issues the tcgen05.mma of query tile t = 0, 1: S_t = Q_t K^T,
+//                   O_t += P_t V; the softmax of one query tile runs under the MMAs of the other;
 //   warps 4-7     : softmax of query tile 0 (thread r owns query row r = tensor-memory lane r):
 //                   mask, running maximum, P = exp2(.), row sum, P (bf16) back into tensor memory;
 //   warps 8-11    : the same for query tile 1;
@@ -35,8 +35,8 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the row max grows by more
 constexpr int kSchedDepth = 2;
-// arrivals that free a queue slot: the MMA thread and one lane of each of the 12 softmax / epilogue warps
-constexpr uint32_t kSchedReaders = 13;
+// arrivals that free a queue slot: the two MMA threads and one lane of each of the 12 softmax / epilogue warps
+constexpr uint32_t kSchedReaders = 14;
 // registers per thread of each role (warpgroups of 128 threads: 72 + 2 * 184 + 72 = 512)
 constexpr uint32_t kRegsControl = 72, kRegsSoftmax = 184, kRegsEpilogue = 72;
 constexpr int kHalfWidthSmem = 128;  // entries of the half-width table kept in shared memory
@@ -62,7 +62,7 @@ struct Ctrl {
     uint64_t kv_full[kRing], kv_empty[kRing];
     uint64_t s_full[2], p_ready[2], o_full[2], o_empty[2], stats_full[2], stats_empty[2];
     uint64_t sched_full[kSchedDepth], sched_empty[kSchedDepth];
-    uint64_t drain;
+    uint64_t drain[2];
     int32_t sched_item[kSchedDepth];            // queue position, >= total: no more work
     int32_t sched_bh[kSchedDepth];
     clear_pair_item_t sched_rec[kSchedDepth];   // the item's record, read once from global memory
@@ -82,7 +82,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1;
-    atomicExch(status, code);
+    atomicCAS(status, 0, code);  // the first wait that expired names the cause
     return false;
 }
 // Drain: wait for a phase regardless of the abort flag (used before leaving with copies in flight).
@@ -166,12 +166,6 @@ __device__ __forceinline__ int step_tile_index(int flags, int side)
     if (side == 0 || (flags & CLEAR_STEP_SHARED)) return 0;
     return (flags & CLEAR_STEP_USE0) ? 1 : 0;
 }
-// Is `side` the last reader of its tile in this step?  (Tile 1 runs after tile 0 within a step.)
-__device__ __forceinline__ bool step_last_reader(int flags, int side)
-{
-    if (!(flags & CLEAR_STEP_SHARED)) return true;
-    return side == 1;
-}
 
 template <int D>
 __global__ void __launch_bounds__(kWsThreads, 1)
@@ -232,13 +226,14 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         }
         for (int i = 0; i < kRing; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->kv_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->kv_empty[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->kv_empty[i]), 2);
         }
         for (int i = 0; i < kSchedDepth; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->sched_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->sched_empty[i]), kSchedReaders);
         }
-        ptx::mbar_init(ptx::smem_u32(&ctrl->drain), 1);
+        ptx::mbar_init(ptx::smem_u32(&ctrl->drain[0]), 1);
+        ptx::mbar_init(ptx::smem_u32(&ctrl->drain[1]), 1);
         ptx::fence_mbar_init();
     }
     for (int i = tid; i < prm.n_half_width && i < kHalfWidthSmem; i += kWsThreads) ctrl->half_width[i] = prm.half_width[i];
@@ -331,16 +326,43 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     drain_bar(ptx::smem_u32(&ctrl->kv_full[idx % kRing]), (idx / kRing) & 1u);
                 }
             }
-        } else if (warp == 1 && lane == 0) {
-            // ================= MMA issuer ================================================================
-            uint32_t ring_base = 0;          // K/V stages consumed by the items before this one
-            uint32_t n_q[2] = {0, 0};        // items seen per query tile
-            uint32_t n_p[2] = {0, 0};        // P tiles consumed per query tile
+        } else if ((warp == 1 || warp == 2) && lane == 0) {
+            // ================= MMA issuer of query tile t: S_t = Q_t K^T, O_t += P_t V ===============
+            // One thread per query tile, so that neither tile waits for the other's softmax; the
+            // tensor core runs each thread's MMAs in the order that thread issued them.
+            const int t = warp - 1;
+            constexpr uint32_t kDescHiK = ptx::smem_desc_hi_sw128(1024);  // 8-row groups are 1024 bytes apart
+            const uint32_t q_lo = ptx::smem_desc_lo(sQ + t * kTileBytes, 16);
+            const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
+            const uint32_t b_sfull = ptx::smem_u32(&ctrl->s_full[t]), b_pready = ptx::smem_u32(&ctrl->p_ready[t]);
+            uint32_t ring_base = 0;  // K/V stages filled by the items before this one
+            uint32_t n_it = 0;       // items in which this query tile existed
+            uint32_t n_p = 0;        // P tiles consumed
             bool ok = true;
+            // Both MMA threads walk EVERY ring position in order and arrive once on its "empty" barrier: with
+            // an MMA commit where they read the stage, at once where they do not.  A stage is refilled only
+            // after both arrivals, so neither thread ever waits on a barrier phase that is more than one
+            // ahead of the barrier (mbarrier waits tell phases apart by one parity bit only).
+            uint32_t next_pos = 0;
             auto kv_wait = [&](uint32_t pos) -> uint32_t {
+                for (; next_pos < pos && ok; ++next_pos) {
+                    const uint32_t st = next_pos % kRing, fl = next_pos / kRing;
+                    ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[st]), fl & 1u, abort_flag, prm.status, 15);
+                    if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->kv_empty[st]));
+                }
                 const uint32_t stage = pos % kRing, fill = pos / kRing;
-                ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[stage]), fill & 1u, abort_flag, prm.status, 4);
+                if (ok) ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[stage]), fill & 1u, abort_flag, prm.status, 4);
+                next_pos = pos + 1;
                 return stage;
+            };
+            auto kv_release = [&](uint32_t stage) { ptx::tc_commit(ptx::smem_u32(&ctrl->kv_empty[stage])); };
+            // walk past every position below `pos` (stages this thread does not read)
+            auto kv_pass_until = [&](uint32_t pos) {
+                for (; next_pos < pos && ok; ++next_pos) {
+                    const uint32_t st = next_pos % kRing, fl = next_pos / kRing;
+                    ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[st]), fl & 1u, abort_flag, prm.status, 15);
+                    if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->kv_empty[st]));
+                }
             };
             for (uint32_t k = 0; ok; ++k) {
                 const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
@@ -349,82 +371,96 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 const clear_pair_item_t item = ctrl->sched_rec[slot];
                 ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
                 if (g >= total_items) break;
+                if (t >= item.n_sides) {
+                    ring_base += (uint32_t)item.n_loads;
+                    kv_pass_until(ring_base);
+                    continue;
+                }
                 const clear_pair_step_t *steps = prm.steps + item.step_begin;
                 const int n = item.step_count;
-                for (int t = 0; t < item.n_sides && ok; ++t)
-                    ok = wait_bar(ptx::smem_u32(&ctrl->q_full[t]), n_q[t] & 1u, abort_flag, prm.status, 6);
+                ok = wait_bar(ptx::smem_u32(&ctrl->q_full[t]), n_it & 1u, abort_flag, prm.status, 6);
                 if (!ok) break;
 
-                // S_t = Q_t K^T for the key tile of `st`
-                auto issue_qk = [&](const clear_pair_step_t &st, int t) {
+                // S_t = Q_t K^T for the key tile of `st`; both operands K-major: 16 contraction channels
+                // are 32 bytes along a 128-byte row, the next 64 channels are the tile's second half
+                auto issue_qk = [&](const clear_pair_step_t &st) {
                     const uint32_t pos = ring_base + (uint32_t)st.load_base + (uint32_t)step_tile_index(st.flags, t);
                     const uint32_t stage = kv_wait(pos);
                     if (!ok) return;
                     ptx::tc_fence_after();
-                    const uint32_t sK = sRing + stage * kTileBytes, sQt = sQ + t * kTileBytes;
+                    const uint32_t k_lo = ptx::smem_desc_lo(sRing + stage * kTileBytes, 16);
+                    ptx::mma_ss_c<false>(tmem_S, ptx::make_desc(q_lo, kDescHiK), ptx::make_desc(k_lo, kDescHiK), kIdescQK);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                        ptx::mma_ss(tmem + t * 128, ptx::smem_desc_sw128(sQt + off, 16, 1024),
-                                    ptx::smem_desc_sw128(sK + off, 16, 1024), kIdescQK, kk > 0);
+                    for (int kk = 1; kk < D / 16; ++kk) {
+                        const uint32_t off16 = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                        ptx::mma_ss_c<true>(tmem_S, ptx::make_desc(q_lo + off16, kDescHiK),
+                                            ptx::make_desc(k_lo + off16, kDescHiK), kIdescQK);
                     }
-                    ptx::tc_commit(ptx::smem_u32(&ctrl->s_full[t]));
-                    if (step_last_reader(st.flags, t)) ptx::tc_commit(ptx::smem_u32(&ctrl->kv_empty[stage]));
+                    ptx::tc_commit(b_sfull);
+                    kv_release(stage);
+                    // stages between this K tile and this tile's V tile belong to the other query tile
+                    kv_pass_until(pos + (uint32_t)step_n_tiles(st.flags));
                 };
 
+                // first step this query tile takes part in (every tile has at least one)
+                int s = 0;
                 clear_pair_step_t cur = load_step(steps);
-                for (int t = 0; t < 2 && ok; ++t)
-                    if (step_uses(cur.flags, t)) issue_qk(cur, t);
-                if (n == 1) {
-                    for (int t = 0; t < item.n_sides; ++t) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
-                }
-                uint32_t n_pv[2] = {0, 0};
-                for (int s = 0; s < n && ok; ++s) {
-                    clear_pair_step_t nxt = cur;
-                    const bool has_next = s + 1 < n;
-                    if (has_next) nxt = load_step(steps + s + 1);
-                    for (int t = 0; t < 2 && ok; ++t) {
-                        if (step_uses(cur.flags, t)) {
-                            // O_t += P_t V
-                            ok = wait_bar(ptx::smem_u32(&ctrl->p_ready[t]), n_p[t] & 1u, abort_flag, prm.status, 7);
-                            if (!ok) break;
-                            ++n_p[t];
-                            const uint32_t pos = ring_base + (uint32_t)cur.load_base + (uint32_t)step_n_tiles(cur.flags) +
-                                                 (uint32_t)step_tile_index(cur.flags, t);
-                            const uint32_t stage = kv_wait(pos);
-                            if (!ok) break;
-                            if (n_pv[t] == 0) {
-                                // the epilogue must have read the previous item's O_t out of tensor memory
-                                ok = wait_bar(ptx::smem_u32(&ctrl->o_empty[t]), (n_q[t] & 1u) ^ 1u, abort_flag, prm.status, 8);
-                                if (!ok) break;
-                            }
-                            ptx::tc_fence_after();
-                            const uint32_t sV = sRing + stage * kTileBytes;
+                while (!step_uses(cur.flags, t) && s + 1 < n) cur = load_step(steps + ++s);
+                clear_pair_step_t pre = cur;  // record s + 1, fetched one step ahead
+                if (s + 1 < n) pre = load_step(steps + s + 1);
+                issue_qk(cur);
+                bool first_pv = true;
+                while (ok) {
+                    // next step of this query tile
+                    int s2 = s + 1;
+                    clear_pair_step_t nxt = pre;
+                    while (s2 < n && !step_uses(nxt.flags, t)) {
+                        ++s2;
+                        if (s2 < n) nxt = load_step(steps + s2);
+                    }
+                    const bool has_next = s2 < n;
+                    if (has_next && s2 + 1 < n) pre = load_step(steps + s2 + 1);
+                    // every Q_t K^T of the item has been issued: the next item's Q tile may land
+                    if (!has_next) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
+
+                    // O_t += P_t V
+                    ok = wait_bar(b_pready, n_p & 1u, abort_flag, prm.status, 7);
+                    if (!ok) break;
+                    ++n_p;
+                    const uint32_t pos = ring_base + (uint32_t)cur.load_base + (uint32_t)step_n_tiles(cur.flags) +
+                                         (uint32_t)step_tile_index(cur.flags, t);
+                    const uint32_t stage = kv_wait(pos);
+                    if (!ok) break;
+                    if (first_pv) {
+                        // the epilogue must have read the previous item's O_t out of tensor memory
+                        ok = wait_bar(ptx::smem_u32(&ctrl->o_empty[t]), (n_it & 1u) ^ 1u, abort_flag, prm.status, 8);
+                        if (!ok) break;
+                    }
+                    ptx::tc_fence_after();
+                    // V is the MN-major operand: 16 keys are 16 rows of 128 bytes = 2048 bytes
+                    const uint32_t v_lo = ptx::smem_desc_lo(sRing + stage * kTileBytes, kHalfBytes);
+                    ptx::mma_ts(tmem_O, tmem_S, ptx::make_desc(v_lo, kDescHiK), kIdescPV, first_pv ? 0u : 1u);
 #pragma unroll
-                            for (int kk = 0; kk < 8; ++kk) {
-                                const uint64_t bdesc = ptx::smem_desc_sw128(sV + kk * 2048, kHalfBytes, 1024);
-                                ptx::mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8, bdesc, kIdescPV,
-                                            (n_pv[t] > 0 || kk > 0) ? 1u : 0u);
-                            }
-                            ++n_pv[t];
-                            if (step_last_reader(cur.flags, t)) ptx::tc_commit(ptx::smem_u32(&ctrl->kv_empty[stage]));
-                        }
-                        if (!has_next && t < item.n_sides) ptx::tc_commit(ptx::smem_u32(&ctrl->o_full[t]));
-                        if (has_next && step_uses(nxt.flags, t)) issue_qk(nxt, t);
+                    for (int kk = 1; kk < 8; ++kk)
+                        ptx::mma_ts_c<true>(tmem_O, tmem_S + kk * 8, ptx::make_desc(v_lo + kk * (2048 >> 4), kDescHiK), kIdescPV);
+                    first_pv = false;
+                    kv_release(stage);
+                    if (!has_next) {
+                        ptx::tc_commit(ptx::smem_u32(&ctrl->o_full[t]));
+                        break;
                     }
-                    if (has_next && s + 2 == n) {
-                        // every Q_t K^T of the item has been issued: the next item's Q tiles may land
-                        for (int t = 0; t < item.n_sides; ++t) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
-                    }
+                    issue_qk(nxt);
                     cur = nxt;
+                    s = s2;
                 }
-                for (int t = 0; t < item.n_sides; ++t) ++n_q[t];
+                ++n_it;
                 ring_base += (uint32_t)item.n_loads;
+                kv_pass_until(ring_base);
             }
             if (*abort_flag) {
                 // MMAs that were issued must retire before tensor memory is given back
-                ptx::tc_commit(ptx::smem_u32(&ctrl->drain));
-                drain_bar(ptx::smem_u32(&ctrl->drain), 0);
+                ptx::tc_commit(ptx::smem_u32(&ctrl->drain[t]));
+                drain_bar(ptx::smem_u32(&ctrl->drain[t]), 0);
             }
         }
         __syncwarp();
