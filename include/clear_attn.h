@@ -111,7 +111,9 @@ enum {
     CLEAR_STEP_SHARED = 4,  /* both visit the SAME key tile (x0, y0): it is staged once             */
     CLEAR_STEP_LINEAR = 8,  /* key tiles of this step are 128 consecutive tokens, else 2-D patches  */
     CLEAR_STEP_MASKED0 = 16, /* tile 0 must apply Eq. 3 / n_valid0 to its key tile                  */
-    CLEAR_STEP_MASKED1 = 32  /* tile 1 likewise                                                     */
+    CLEAR_STEP_MASKED1 = 32, /* tile 1 likewise                                                     */
+    CLEAR_STEP_CLIP0 = 64,   /* tile 0's 2-D key patch reaches past the grid border: such keys do not exist */
+    CLEAR_STEP_CLIP1 = 128   /* tile 1's likewise                                                    */
 };
 
 /* One step of a pair item: each query tile of the pair multiplies against one key tile. */
@@ -119,8 +121,8 @@ typedef struct clear_pair_step {
     int32_t x0, y0;     /* key tile of query tile 0 (and of tile 1 when SHARED); as clear_kv_tile_t */
     int32_t x1, y1;     /* key tile of query tile 1 when not SHARED                                 */
     int32_t flags;      /* CLEAR_STEP_* bits                                                        */
-    int32_t n_valid0;   /* linear tiles: keys [0, n_valid) of the tile exist / are allowed          */
-    int32_t n_valid1;
+    int32_t n_valid0;   /* linear tiles: keys [0, n_valid) of the tile exist / are allowed; 2-D patches: */
+    int32_t n_valid1;   /*   index of the tile pair's entry in the mask table, or -1 if it has none      */
     int32_t load_base;  /* key/value tiles the item has staged before this step (K and V counted
                            separately): position of this step's first stage in the block's ring     */
 } clear_pair_step_t;
@@ -180,6 +182,12 @@ int clear_plan_tables(const clear_plan_t *plan, const clear_work_item_t **items,
  * lists first) and their steps.  Empty for other plans.  Errors: INVALID_ARG. */
 int clear_plan_pair_tables(const clear_plan_t *plan, const clear_pair_item_t **items, int32_t *n_items,
                            const clear_pair_step_t **steps, int32_t *n_steps);
+
+/* Mask table of a TCGEN05_WS plan: Eq. 3 evaluated once per relative position of a key patch to a query
+ * patch (the mask depends only on that offset).  Entry e is 128 rows (queries of the patch, row-major)
+ * of four 32-bit words; bit j of word w tells whether key 32 w + j of the patch (row-major) lies within
+ * the radius of that query.  Grid clipping is not part of it (CLEAR_STEP_CLIP*).  Errors: INVALID_ARG. */
+int clear_plan_mask_table(const clear_plan_t *plan, const uint32_t **words, int32_t *n_entries);
 
 /* Forward pass with an explicit plan.  Tensor dtype is the plan's.  Calls on one plan share its
  * workspace: run them on one stream, or order them yourself.

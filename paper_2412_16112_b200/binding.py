@@ -20,13 +20,14 @@ BF16, F32 = 0, 1
 KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_TCGEN05_WS = 0, 1, 2, 3
 TILE_LINEAR, TILE_MASKED = 1, 2
 STEP_USE0, STEP_USE1, STEP_SHARED, STEP_LINEAR, STEP_MASKED0, STEP_MASKED1 = 1, 2, 4, 8, 16, 32
+STEP_CLIP0, STEP_CLIP1 = 64, 128
 
 EXPORTS = [
     "clear_attn_fwd", "clear_attn_fwd_f32", "clear_plan_create", "clear_plan_create_host",
     "clear_plan_tables", "clear_attn_fwd_planned", "clear_attn_fwd_host", "clear_plan_info",
     "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
     "clear_last_cuda_error", "clear_attn_fwd_static", "clear_plan_pair_tables",
-    "clear_last_device_status",
+    "clear_last_device_status", "clear_plan_mask_table",
 ]
 
 
@@ -100,6 +101,8 @@ def load() -> ctypes.CDLL:
                                                ctypes.POINTER(ctypes.c_int32),
                                                ctypes.POINTER(ctypes.POINTER(PairStep)),
                                                ctypes.POINTER(ctypes.c_int32)]
+        lib.clear_plan_mask_table.argtypes = [vp, ctypes.POINTER(ctypes.POINTER(ctypes.c_uint32)),
+                                              ctypes.POINTER(ctypes.c_int32)]
         lib.clear_attn_fwd_planned.argtypes = [vp, vp, vp, vp, vp, f32, vp]
         lib.clear_attn_fwd_host.argtypes = [vp, vp, vp, vp, vp, f32, vp]
         lib.clear_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
@@ -224,6 +227,15 @@ class Plan:
         _check(load().clear_plan_pair_tables(self._h, ctypes.byref(items), ctypes.byref(ni), ctypes.byref(steps),
                                              ctypes.byref(ns)), "clear_plan_pair_tables")
         return [items[i] for i in range(ni.value)], [steps[i] for i in range(ns.value)]
+
+    def mask_table(self):
+        """Mask table of a TCGEN05_WS plan as a numpy array [n_entries, 128, 4] of uint32 (a copy)."""
+        import numpy as np
+        words, n = ctypes.POINTER(ctypes.c_uint32)(), ctypes.c_int32()
+        _check(load().clear_plan_mask_table(self._h, ctypes.byref(words), ctypes.byref(n)), "clear_plan_mask_table")
+        if n.value == 0:
+            return np.zeros((0, 128, 4), dtype=np.uint32)
+        return np.ctypeslib.as_array(words, shape=(n.value, 128, 4)).copy()
 
     def forward(self, q, k, v, out, scale, stream=None):
         ptrs = _tensor_args(q, k, v, out, self.dtype)

@@ -47,6 +47,7 @@ int free_device_parts(clear_plan *p)
     rel(p->d_tiles);
     rel(p->d_pair_items);
     rel(p->d_pair_steps);
+    rel(p->d_mask_table);
     rel(p->d_status);
     rel(p->d_partial_o);
     rel(p->d_partial_ml);
@@ -59,6 +60,7 @@ int free_device_parts(clear_plan *p)
     p->d_tiles = nullptr;
     p->d_pair_items = nullptr;
     p->d_pair_steps = nullptr;
+    p->d_mask_table = nullptr;
     p->d_status = nullptr;
     p->d_partial_o = nullptr;
     p->d_partial_ml = nullptr;
@@ -104,6 +106,7 @@ int create_plan(clear_plan_t **out, const Shape &shape_in, bool host_only)
         if (rc == CLEAR_OK) rc = upload(&p->d_tiles, p->sch.tiles);
         if (rc == CLEAR_OK) rc = upload(&p->d_pair_items, p->sch.pair_items);
         if (rc == CLEAR_OK) rc = upload(&p->d_pair_steps, p->sch.pair_steps);
+        if (rc == CLEAR_OK) rc = upload(&p->d_mask_table, p->sch.mask_table);
         if (rc == CLEAR_OK) {
             cudaError_t e = cudaMalloc((void **)&p->d_status, kStatusWords * sizeof(int));
             if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, kStatusWords * sizeof(int));
@@ -251,6 +254,14 @@ int clear_plan_pair_tables(const clear_plan_t *plan, const clear_pair_item_t **i
     if (n_items) *n_items = (int32_t)plan->sch.pair_items.size();
     if (steps) *steps = plan->sch.pair_steps.data();
     if (n_steps) *n_steps = (int32_t)plan->sch.pair_steps.size();
+    return CLEAR_OK;
+}
+
+int clear_plan_mask_table(const clear_plan_t *plan, const uint32_t **words, int32_t *n_entries)
+{
+    if (!plan) return CLEAR_ERR_INVALID_ARG;
+    if (words) *words = plan->sch.mask_table.data();
+    if (n_entries) *n_entries = (int32_t)(plan->sch.mask_table.size() / ((size_t)kTileTokens * 4));
     return CLEAR_OK;
 }
 

@@ -21,6 +21,7 @@ struct clear_plan {
     clear_kv_tile_t *d_tiles = nullptr;
     clear_pair_item_t *d_pair_items = nullptr;
     clear_pair_step_t *d_pair_steps = nullptr;
+    uint32_t *d_mask_table = nullptr;
     // [0] status word: 0 = fine, set by a kernel whose bounded wait expired;
     // [1] work-queue head and [2] finished-block count of the persistent kernel (both back at zero
     // when a launch ends)

@@ -4,6 +4,8 @@
 
 #include <algorithm>
 #include <cmath>
+#include <map>
+#include <utility>
 
 namespace clear {
 
@@ -172,6 +174,7 @@ namespace {
 struct PatchTile {
     int x, y;
     bool masked;
+    bool clipped;  // part of the patch lies outside the grid
 };
 
 // Key patches (on the 8 x 16 lattice) that hold at least one key allowed to some query of the patch
@@ -194,7 +197,7 @@ std::vector<PatchTile> patches_of(const Shape &s, int64_t thr, int R, int qx, in
             const int64_t fx = std::max(kx1 - qx, qx1 - bx);
             const int64_t fy = std::max(ky1 - qy, qy1 - by);
             const bool whole = (bx + kTileW <= gw) && (by + kTileH <= gh);
-            out.push_back(PatchTile{bx, by, !(whole && fx * fx + fy * fy < thr)});
+            out.push_back(PatchTile{bx, by, !(whole && fx * fx + fy * fy < thr), !whole});
         }
     }
     return out;
@@ -212,6 +215,27 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
 
     sch.pair_items.clear();
     sch.pair_steps.clear();
+    sch.mask_table.clear();
+
+    // Eq. 3 for a key patch at offset (dy, dx) from a query patch, once per distinct offset
+    std::map<std::pair<int, int>, int> mask_ids;
+    auto mask_entry = [&](int dy, int dx) -> int {
+        auto it = mask_ids.find({dy, dx});
+        if (it != mask_ids.end()) return it->second;
+        if ((int)mask_ids.size() >= kMaxMaskEntries) return -1;
+        const int id = (int)mask_ids.size();
+        mask_ids[{dy, dx}] = id;
+        sch.mask_table.resize((size_t)(id + 1) * kTileTokens * 4, 0u);
+        uint32_t *e = sch.mask_table.data() + (size_t)id * kTileTokens * 4;
+        for (int r = 0; r < kTileTokens; ++r) {
+            const int qy = r / kTileW, qx = r % kTileW;
+            for (int j = 0; j < kTileTokens; ++j) {
+                const int64_t ddy = dy + j / kTileW - qy, ddx = dx + j % kTileW - qx;
+                if (ddx * ddx + ddy * ddy < thr) e[r * 4 + (j >> 5)] |= 1u << (j & 31);
+            }
+        }
+        return id;
+    };
 
     auto finish_item = [&](clear_pair_item_t &it) {
         int32_t loads = 0;
@@ -315,12 +339,16 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
                 if (i < only_a.size()) {
                     st.x0 = only_a[i].x;
                     st.y0 = only_a[i].y;
-                    st.flags |= CLEAR_STEP_USE0 | (only_a[i].masked ? CLEAR_STEP_MASKED0 : 0);
+                    st.flags |= CLEAR_STEP_USE0 | (only_a[i].masked ? CLEAR_STEP_MASKED0 : 0) |
+                                (only_a[i].clipped ? CLEAR_STEP_CLIP0 : 0);
+                    st.n_valid0 = only_a[i].masked ? mask_entry(st.y0 - it.qy0, st.x0 - it.qx) : -1;
                 }
                 if (i < only_b.size()) {
                     st.x1 = only_b[i].x;
                     st.y1 = only_b[i].y;
-                    st.flags |= CLEAR_STEP_USE1 | (only_b[i].masked ? CLEAR_STEP_MASKED1 : 0);
+                    st.flags |= CLEAR_STEP_USE1 | (only_b[i].masked ? CLEAR_STEP_MASKED1 : 0) |
+                                (only_b[i].clipped ? CLEAR_STEP_CLIP1 : 0);
+                    st.n_valid1 = only_b[i].masked ? mask_entry(st.y1 - it.qy1, st.x1 - it.qx) : -1;
                 }
                 sch.pair_steps.push_back(st);
             }
@@ -330,7 +358,10 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
                 st.x0 = st.x1 = ab.first.x;
                 st.y0 = st.y1 = ab.first.y;
                 st.flags = CLEAR_STEP_USE0 | CLEAR_STEP_USE1 | CLEAR_STEP_SHARED |
-                           (ab.first.masked ? CLEAR_STEP_MASKED0 : 0) | (ab.second.masked ? CLEAR_STEP_MASKED1 : 0);
+                           (ab.first.masked ? CLEAR_STEP_MASKED0 : 0) | (ab.second.masked ? CLEAR_STEP_MASKED1 : 0) |
+                           (ab.first.clipped ? (CLEAR_STEP_CLIP0 | CLEAR_STEP_CLIP1) : 0);
+                st.n_valid0 = ab.first.masked ? mask_entry(st.y0 - it.qy0, st.x0 - it.qx) : -1;
+                st.n_valid1 = ab.second.masked ? mask_entry(st.y1 - it.qy1, st.x1 - it.qx) : -1;
                 sch.pair_steps.push_back(st);
             }
             finish_item(it);

@@ -12,6 +12,7 @@ constexpr int kTileH = 8;      // query / key patch: 8 grid rows ...
 constexpr int kTileW = 16;     // ... by 16 grid columns = 128 tokens
 constexpr int kTileTokens = 128;
 constexpr int kSplitTargetTiles = 64;  // key tiles per split of a text-query tile
+constexpr int kMaxMaskEntries = 512;   // relative patch offsets with a precomputed mask (2 KB each)
 
 struct Shape {
     int B = 0, H = 0, grid_h = 0, grid_w = 0, n_text = 0, head_dim = 0;
@@ -33,6 +34,7 @@ struct Schedule {
     std::vector<clear_pair_item_t> pair_items;   // TCGEN05_WS: text items first, then image items
     std::vector<clear_pair_step_t> pair_steps;
     int n_text_pair_items = 0;
+    std::vector<uint32_t> mask_table;            // TCGEN05_WS: [entry][128 query rows][4 words]
     int n_text_tiles = 0;                // text-query tiles of 128 rows
     int n_text_splits = 0;               // splits per text-query tile (1 = no partial results)
     int n_partial_slots = 0;

@@ -45,6 +45,7 @@ struct WsParams {
     const clear_pair_item_t *items;
     const clear_pair_step_t *steps;
     const int32_t *half_width;
+    const uint32_t *mask_table;  // [entry][128 query rows][4 words]: Eq. 3 per relative patch offset
     int n_half_width;
     int grid_h, grid_w, n_text;
     long long n_tokens;
@@ -501,13 +502,26 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
 
+            // Step records are fetched two steps ahead and this row's precomputed mask words one step
+            // ahead, so that neither latency is on the critical path.
+            const int kMaskedBit = t ? CLEAR_STEP_MASKED1 : CLEAR_STEP_MASKED0;
+            auto load_mask_row = [&](const SideStep &q) -> uint4 {
+                if (step_uses(q.flags, t) && (q.flags & kMaskedBit) && !(q.flags & CLEAR_STEP_LINEAR) && q.n_valid >= 0)
+                    return __ldg(reinterpret_cast<const uint4 *>(prm.mask_table) + ((size_t)q.n_valid * 128 + r));
+                return make_uint4(0u, 0u, 0u, 0u);
+            };
             SideStep st_next = load_side_step(steps, t);
+            SideStep st_next2 = st_next;
+            if (item.step_count > 1) st_next2 = load_side_step(steps + 1, t);
+            uint4 mrow_next = load_mask_row(st_next);
             for (int s = 0; s < item.step_count; ++s) {
-                // the next record is fetched one step ahead, so its latency is off the critical path
                 const SideStep st = st_next;
-                if (s + 1 < item.step_count) st_next = load_side_step(steps + s + 1, t);
+                const uint4 mrow = mrow_next;
+                st_next = st_next2;
+                if (s + 2 < item.step_count) st_next2 = load_side_step(steps + s + 2, t);
+                if (s + 1 < item.step_count) mrow_next = load_mask_row(st_next);
                 if (!step_uses(st.flags, t)) continue;
-                const bool masked = (st.flags & (t ? CLEAR_STEP_MASKED1 : CLEAR_STEP_MASKED0)) != 0;
+                const bool masked = (st.flags & kMaskedBit) != 0;
                 // ---- mask bits of this row for the tile (bit j = key j allowed) -----------------------
                 uint32_t mw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
                 if (masked) {
@@ -516,6 +530,23 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         for (int w = 0; w < 4; ++w) {
                             const int nv = min(max(st.n_valid - 32 * w, 0), 32);
                             mw[w] = nv == 32 ? 0xffffffffu : ((1u << nv) - 1u);
+                        }
+                    } else if (st.n_valid >= 0) {
+                        // Eq. 3 from the table; keys of the patch that lie off the grid do not exist
+                        mw[0] = mrow.x;
+                        mw[1] = mrow.y;
+                        mw[2] = mrow.z;
+                        mw[3] = mrow.w;
+                        if (st.flags & (t ? CLEAR_STEP_CLIP1 : CLEAR_STEP_CLIP0)) {
+                            const int lo = max(0, -st.x), hi = min(15, prm.grid_w - 1 - st.x);
+                            const uint32_t cols = lo <= hi ? (((1u << (hi - lo + 1)) - 1u) << lo) : 0u;
+#pragma unroll
+                            for (int w = 0; w < 4; ++w) {
+                                const int ky0 = st.y + 2 * w, ky1 = ky0 + 1;
+                                const uint32_t ok0 = (ky0 >= 0 && ky0 < prm.grid_h) ? cols : 0u;
+                                const uint32_t ok1 = (ky1 >= 0 && ky1 < prm.grid_h) ? cols : 0u;
+                                mw[w] &= ok0 | (ok1 << 16);
+                            }
                         }
                     } else {
 #pragma unroll
@@ -548,19 +579,31 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 for (int w = 0; w < 4; ++w) ptx::tmem_ld32(tmem_S + lane_off + 32 * w, sv[w]);
                 ptx::tmem_wait_ld();
 
+                // Groups of 16 keys (one grid row of a key patch) that no query of this warp may see are
+                // skipped altogether: bit g of `live` = some lane has an allowed key in group g.
+                uint32_t live = 0xffu;
+                if (masked) {
+                    live = 0u;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        if (__any_sync(0xffffffffu, ((mw[g >> 1] >> (16 * (g & 1))) & 0xffffu) != 0u)) live |= 1u << g;
+                }
                 // row maximum over the allowed keys, four independent chains of three-input maxima
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 if (masked) {
 #pragma unroll
-                    for (int w = 0; w < 4; ++w)
+                    for (int g = 0; g < 8; ++g) {
+                        if (!(live & (1u << g))) continue;
+                        const int w = g >> 1;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
+                        for (int j = 16 * (g & 1); j < 16 * (g & 1) + 16; j += 2) {
                             const float v0 = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
                             const float v1 = ((mw[w] >> (j + 1)) & 1u) ? __uint_as_float(sv[w][j + 1]) : -INFINITY;
                             sv[w][j] = __float_as_uint(v0);
                             sv[w][j + 1] = __float_as_uint(v1);
                             mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], v0, v1);
                         }
+                    }
                 } else {
 #pragma unroll
                     for (int w = 0; w < 4; ++w)
@@ -606,13 +649,22 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 for (int w = 0; w < 4; ++w) {
                     uint32_t pk[16];
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        const uint64_t x2 = ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
-                        float x0, x1;
-                        ptx::unpack2(x2, x0, x1);
-                        const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
-                        lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
-                        pk[j >> 1] = ptx::pack_bf16(p0, p1);
+                    for (int hh = 0; hh < 2; ++hh) {
+                        if (live & (1u << (2 * w + hh))) {
+#pragma unroll
+                            for (int j = 16 * hh; j < 16 * hh + 16; j += 2) {
+                                const uint64_t x2 =
+                                    ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
+                                float x0, x1;
+                                ptx::unpack2(x2, x0, x1);
+                                const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
+                                lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
+                                pk[j >> 1] = ptx::pack_bf16(p0, p1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 8 * hh; j < 8 * hh + 8; ++j) pk[j] = 0u;
+                        }
                     }
                     ptx::tmem_st16(tmem_S + lane_off + 16 * w, pk);
                 }
@@ -870,6 +922,7 @@ int launch_ws(const clear_plan &p, const void *q, const void *k, const void *v, 
     prm.items = p.d_pair_items;
     prm.steps = p.d_pair_steps;
     prm.half_width = p.d_half_width;
+    prm.mask_table = p.d_mask_table;
     prm.n_half_width = (int)p.sch.half_width.size();
     prm.grid_h = p.shape.grid_h;
     prm.grid_w = p.shape.grid_w;

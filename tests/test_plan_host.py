@@ -197,6 +197,38 @@ def key_tokens(x, y, linear, n_valid, gh, gw, T, th, tw):
     return (T + ys * gw + xs)[ok], bool(ok.all())
 
 
+def check_mask_table(p, items, steps, gh, gw, T, r, th, tw):
+    """Every masked 2-D tile's table entry, restricted to the keys on the grid, is the oracle's mask;
+    the clip flag is set exactly when part of the key patch is off the grid."""
+    table = p.mask_table()
+    for it in items:
+        if it.kind != 0:
+            continue
+        for st in steps[it.step_begin: it.step_begin + it.step_count]:
+            if st.flags & clear.STEP_LINEAR:
+                continue
+            for side in range(it.n_sides):
+                if not st.flags & (clear.STEP_USE1 if side else clear.STEP_USE0):
+                    continue
+                x, y, e = (st.x1, st.y1, st.n_valid1) if side else (st.x0, st.y0, st.n_valid0)
+                qy = it.qy1 if side else it.qy0
+                ys, xs = np.meshgrid(np.arange(y, y + th), np.arange(x, x + tw), indexing="ij")
+                on_grid = ((ys >= 0) & (ys < gh) & (xs >= 0) & (xs < gw)).reshape(-1)
+                clip = bool(st.flags & (clear.STEP_CLIP1 if side else clear.STEP_CLIP0))
+                assert clip == (not on_grid.all())
+                if not st.flags & (clear.STEP_MASKED1 if side else clear.STEP_MASKED0):
+                    continue
+                assert 0 <= e < len(table), "masked 2-D tile without a mask-table entry"
+                bits = ((table[e][:, :, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(128, 128).astype(bool)
+                toks = (T + ys * gw + xs).reshape(-1)
+                for rr in range(128):
+                    q_y, q_x = qy + rr // tw, it.qx + rr % tw
+                    if q_y >= gh or q_x >= gw:
+                        continue
+                    row = oracle.mask_row(T + q_y * gw + q_x, gh, gw, T, r).astype(bool)
+                    assert np.array_equal(bits[rr][on_grid], row[toks[on_grid]])
+
+
 @pytest.mark.parametrize("gh,gw,T,r", SHAPES + [(40, 40, 300, 9.0), (17, 16, 129, 4.0)])
 def test_pair_schedule_covers_each_allowed_pair_exactly_once(gh, gw, T, r):
     p = clear.Plan(1, 1, gh, gw, T, 128, r, kernel=clear.KERNEL_TCGEN05_WS, host_only=True)
@@ -285,6 +317,7 @@ def test_pair_schedule_covers_each_allowed_pair_exactly_once(gh, gw, T, r):
                 assert rows[q][unmasked].all(), "a tile flagged mask-free holds a disallowed pair"
     assert info.executed_pairs == executed
     assert np.all(seen_queries[T:] == 1)
+    check_mask_table(p, items, steps, gh, gw, T, r, th, tw)
     for q0 in range(0, T, 128):
         assert sorted(text_cover[q0]) == list(range(N))
     if info.n_text_splits > 1:
