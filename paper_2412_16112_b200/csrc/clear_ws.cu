@@ -14,8 +14,10 @@
 //   warps 8-11    : the same for query tile 1;
 //   warps 12-15   : epilogue: O / l -> bf16 -> global memory (or fp32 partial results of split
 //                   text rows), while the other warps already run the next item.
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each; P overwrites S in place.
-// Shared memory: Q0, Q1 and a ring of five key/value stages (K and V tiles take one stage each).
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each.  P goes through shared memory, 64
+// keys at a time, so that S_t of the next step can be computed while the softmax of this one runs.
+// Shared memory: Q0, Q1, a ring of four key/value stages (K and V tiles take one stage each) and one
+// half-tile of P per query tile.
 // Every wait is bounded: on expiry the block raises the plan's status word and leaves.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -30,9 +32,11 @@ namespace clear {
 namespace {
 
 constexpr int kWsThreads = 512;
-constexpr int kRing = 5;
+constexpr int kRing = 4;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kWaitHintNs = 20000;            // one sleep inside try_wait
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the row max grows by more
 constexpr int kSchedDepth = 2;
 // arrivals that free a queue slot: the two MMA threads and one lane of each of the 12 softmax / epilogue warps
@@ -61,7 +65,7 @@ struct WsParams {
 struct Ctrl {
     uint64_t q_full[2], q_empty[2];
     uint64_t kv_full[kRing], kv_empty[kRing];
-    uint64_t s_full[2], p_ready[2], o_full[2], o_empty[2], stats_full[2], stats_empty[2];
+    uint64_t s_full[2], s_free[2], p_ready[2][2], p_free[2], o_full[2], o_empty[2], stats_full[2], stats_empty[2];
     uint64_t sched_full[kSchedDepth], sched_empty[kSchedDepth];
     uint64_t drain[2];
     int32_t sched_item[kSchedDepth];            // queue position, >= total: no more work
@@ -74,17 +78,25 @@ struct Ctrl {
     int32_t half_width[kHalfWidthSmem];
 };
 
-// Bounded wait on an mbarrier phase.  Returns false once the block has given up.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+// Bounded wait on an mbarrier phase.  Returns false once the block has given up.  A waiting thread
+// sleeps inside try_wait (suspend-time hint) rather than spinning: a spinning warp would take issue
+// slots and instruction-cache lines from the softmax warps of its scheduler.
+__device__ __forceinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if (it > 256) __nanosleep(it > 8192 ? 256 : 32);
-        if ((it & 255u) == 255u && *abort_flag) return false;
+    const uint64_t t0 = ptx::globaltimer_ns();
+    for (;;) {
+        if (ptx::mbar_try_wait_hint(bar, parity, kWaitHintNs)) return true;
+        if (*abort_flag) return false;
+        if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) break;
     }
     *abort_flag = 1;
     atomicCAS(status, 0, code);  // the first wait that expired names the cause
     return false;
+}
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    return wait_bar_slow(bar, parity, abort_flag, status, code);
 }
 // Drain: wait for a phase regardless of the abort flag (used before leaving with copies in flight).
 __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity)
@@ -183,8 +195,10 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t smem_base = ptx::smem_u32(smem_raw);
-    const uint32_t sQ = smem_base, sRing = sQ + 2 * kTileBytes;
-    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_raw + (2 + kRing) * kTileBytes);
+    // Q0, Q1 | ring of K/V stages | one half-tile of P (128 queries x 64 keys) per query tile | control
+    const uint32_t sQ = smem_base, sRing = sQ + 2 * kTileBytes, sP = sRing + kRing * kTileBytes;
+    constexpr uint32_t kCtrlOff = (2 + kRing) * kTileBytes + 2 * kHalfBytes;
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_raw + kCtrlOff);
     volatile int *abort_flag = &ctrl->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -219,7 +233,10 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_empty[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->s_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->s_free[i]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][0]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][1]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_free[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->o_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 128);
             ptx::mbar_init(ptx::smem_u32(&ctrl->stats_full[i]), 128);
@@ -331,40 +348,45 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             // ================= MMA issuer of query tile t: S_t = Q_t K^T, O_t += P_t V ===============
             // One thread per query tile, so that neither tile waits for the other's softmax; the
             // tensor core runs each thread's MMAs in the order that thread issued them.
+            // S_t(next) is issued as soon as the softmax warps have taken S_t into registers, i.e.
+            // before P_t V of the current step: P travels through shared memory, in two halves of 64 keys.
             const int t = warp - 1;
             constexpr uint32_t kDescHiK = ptx::smem_desc_hi_sw128(1024);  // 8-row groups are 1024 bytes apart
             const uint32_t q_lo = ptx::smem_desc_lo(sQ + t * kTileBytes, 16);
+            const uint32_t p_lo = ptx::smem_desc_lo(sP + t * kHalfBytes, 16);
             const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
-            const uint32_t b_sfull = ptx::smem_u32(&ctrl->s_full[t]), b_pready = ptx::smem_u32(&ctrl->p_ready[t]);
+            const uint32_t b_sfull = ptx::smem_u32(&ctrl->s_full[t]), b_sfree = ptx::smem_u32(&ctrl->s_free[t]);
+            const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]);
             uint32_t ring_base = 0;  // K/V stages filled by the items before this one
             uint32_t n_it = 0;       // items in which this query tile existed
-            uint32_t n_p = 0;        // P tiles consumed
+            uint32_t n_qk = 0;       // S tiles issued
+            uint32_t n_pv = 0;       // steps whose P V has been issued
             bool ok = true;
             // Both MMA threads walk EVERY ring position in order and arrive once on its "empty" barrier: with
             // an MMA commit where they read the stage, at once where they do not.  A stage is refilled only
             // after both arrivals, so neither thread ever waits on a barrier phase that is more than one
             // ahead of the barrier (mbarrier waits tell phases apart by one parity bit only).
-            uint32_t next_pos = 0;
-            auto kv_wait = [&](uint32_t pos) -> uint32_t {
+            uint32_t next_pos = 0;  // first position whose fill this thread has not seen yet
+            // see the fills of [next_pos, pos) and free them at once, except `keep` (a V tile still to be read)
+            auto kv_walk = [&](uint32_t pos, uint32_t keep) {
                 for (; next_pos < pos && ok; ++next_pos) {
                     const uint32_t st = next_pos % kRing, fl = next_pos / kRing;
                     ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[st]), fl & 1u, abort_flag, prm.status, 15);
-                    if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->kv_empty[st]));
+                    if (ok && next_pos != keep) ptx::mbar_arrive(ptx::smem_u32(&ctrl->kv_empty[st]));
                 }
+            };
+            // wait for the fill of `pos`, a stage this thread reads
+            auto kv_wait = [&](uint32_t pos, uint32_t keep) -> uint32_t {
+                kv_walk(pos, keep);
                 const uint32_t stage = pos % kRing, fill = pos / kRing;
-                if (ok) ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[stage]), fill & 1u, abort_flag, prm.status, 4);
-                next_pos = pos + 1;
+                if (ok && next_pos == pos) {
+                    ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[stage]), fill & 1u, abort_flag, prm.status, 4);
+                    next_pos = pos + 1;
+                }
                 return stage;
             };
             auto kv_release = [&](uint32_t stage) { ptx::tc_commit(ptx::smem_u32(&ctrl->kv_empty[stage])); };
-            // walk past every position below `pos` (stages this thread does not read)
-            auto kv_pass_until = [&](uint32_t pos) {
-                for (; next_pos < pos && ok; ++next_pos) {
-                    const uint32_t st = next_pos % kRing, fl = next_pos / kRing;
-                    ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[st]), fl & 1u, abort_flag, prm.status, 15);
-                    if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->kv_empty[st]));
-                }
-            };
+            constexpr uint32_t kNone = 0xffffffffu;
             for (uint32_t k = 0; ok; ++k) {
                 const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
                 if (!wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 5)) break;
@@ -374,7 +396,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 if (g >= total_items) break;
                 if (t >= item.n_sides) {
                     ring_base += (uint32_t)item.n_loads;
-                    kv_pass_until(ring_base);
+                    kv_walk(ring_base, kNone);
                     continue;
                 }
                 const clear_pair_step_t *steps = prm.steps + item.step_begin;
@@ -383,10 +405,14 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 if (!ok) break;
 
                 // S_t = Q_t K^T for the key tile of `st`; both operands K-major: 16 contraction channels
-                // are 32 bytes along a 128-byte row, the next 64 channels are the tile's second half
-                auto issue_qk = [&](const clear_pair_step_t &st) {
+                // are 32 bytes along a 128-byte row, the next 64 channels are the tile's second half.
+                // `keep`: position of a V tile this thread still has to read (or kNone).
+                auto issue_qk = [&](const clear_pair_step_t &st, uint32_t keep) {
+                    // the softmax warps must have taken the previous S_t out of tensor memory
+                    if (n_qk > 0) ok = wait_bar(b_sfree, (n_qk - 1) & 1u, abort_flag, prm.status, 16);
+                    if (!ok) return;
                     const uint32_t pos = ring_base + (uint32_t)st.load_base + (uint32_t)step_tile_index(st.flags, t);
-                    const uint32_t stage = kv_wait(pos);
+                    const uint32_t stage = kv_wait(pos, keep);
                     if (!ok) return;
                     ptx::tc_fence_after();
                     const uint32_t k_lo = ptx::smem_desc_lo(sRing + stage * kTileBytes, 16);
@@ -399,8 +425,11 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     }
                     ptx::tc_commit(b_sfull);
                     kv_release(stage);
-                    // stages between this K tile and this tile's V tile belong to the other query tile
-                    kv_pass_until(pos + (uint32_t)step_n_tiles(st.flags));
+                    ++n_qk;
+                };
+                auto v_position = [&](const clear_pair_step_t &st) -> uint32_t {
+                    return ring_base + (uint32_t)st.load_base + (uint32_t)step_n_tiles(st.flags) +
+                           (uint32_t)step_tile_index(st.flags, t);
                 };
 
                 // first step this query tile takes part in (every tile has at least one)
@@ -409,7 +438,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 while (!step_uses(cur.flags, t) && s + 1 < n) cur = load_step(steps + ++s);
                 clear_pair_step_t pre = cur;  // record s + 1, fetched one step ahead
                 if (s + 1 < n) pre = load_step(steps + s + 1);
-                issue_qk(cur);
+                issue_qk(cur, kNone);
                 bool first_pv = true;
                 while (ok) {
                     // next step of this query tile
@@ -424,39 +453,63 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     // every Q_t K^T of the item has been issued: the next item's Q tile may land
                     if (!has_next) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
 
-                    // O_t += P_t V
-                    ok = wait_bar(b_pready, n_p & 1u, abort_flag, prm.status, 7);
-                    if (!ok) break;
-                    ++n_p;
-                    const uint32_t pos = ring_base + (uint32_t)cur.load_base + (uint32_t)step_n_tiles(cur.flags) +
-                                         (uint32_t)step_tile_index(cur.flags, t);
-                    const uint32_t stage = kv_wait(pos);
-                    if (!ok) break;
-                    if (first_pv) {
-                        // the epilogue must have read the previous item's O_t out of tensor memory
-                        ok = wait_bar(ptx::smem_u32(&ctrl->o_empty[t]), (n_it & 1u) ^ 1u, abort_flag, prm.status, 8);
-                        if (!ok) break;
+                    const uint32_t pos_v = v_position(cur);
+                    // The next S_t goes ahead of this step's P_t V when its K tile sits right behind this V
+                    // tile in the ring; a V tile held back for longer would stall the ring.
+                    bool qk_done = false;
+                    if (has_next) {
+                        const uint32_t pos_k = ring_base + (uint32_t)nxt.load_base + (uint32_t)step_tile_index(nxt.flags, t);
+                        if (pos_k - pos_v <= 2u) {
+                            issue_qk(nxt, pos_v);
+                            qk_done = true;
+                            if (!ok) break;
+                        }
                     }
-                    ptx::tc_fence_after();
-                    // V is the MN-major operand: 16 keys are 16 rows of 128 bytes = 2048 bytes
-                    const uint32_t v_lo = ptx::smem_desc_lo(sRing + stage * kTileBytes, kHalfBytes);
-                    ptx::mma_ts(tmem_O, tmem_S, ptx::make_desc(v_lo, kDescHiK), kIdescPV, first_pv ? 0u : 1u);
+
+                    // O_t += P_t V, 64 keys at a time as the softmax warps deliver P's halves
+                    if (!qk_done) kv_walk(pos_v, kNone);
+                    uint32_t stage_v = 0;
 #pragma unroll
-                    for (int kk = 1; kk < 8; ++kk)
-                        ptx::mma_ts_c<true>(tmem_O, tmem_S + kk * 8, ptx::make_desc(v_lo + kk * (2048 >> 4), kDescHiK), kIdescPV);
+                    for (int h = 0; h < 2; ++h) {
+                        ok = wait_bar(ptx::smem_u32(&ctrl->p_ready[t][h]), n_pv & 1u, abort_flag, prm.status, 7);
+                        if (!ok) break;
+                        if (h == 0) {
+                            stage_v = kv_wait(pos_v, kNone);
+                            if (!ok) break;
+                            if (first_pv) {
+                                // the epilogue must have read the previous item's O_t out of tensor memory
+                                ok = wait_bar(ptx::smem_u32(&ctrl->o_empty[t]), (n_it & 1u) ^ 1u, abort_flag, prm.status, 8);
+                                if (!ok) break;
+                            }
+                        }
+                        ptx::tc_fence_after();
+                        // P half: K-major, 16 keys are 32 bytes along a row; V: MN-major, 16 keys are 16
+                        // rows of 128 bytes = 2048 bytes
+                        const uint32_t v_lo = ptx::smem_desc_lo(sRing + stage_v * kTileBytes, kHalfBytes) + h * 4 * (2048 >> 4);
+                        ptx::mma_ss(tmem_O, ptx::make_desc(p_lo, kDescHiK), ptx::make_desc(v_lo, kDescHiK), kIdescPV,
+                                    (first_pv && h == 0) ? 0u : 1u);
+#pragma unroll
+                        for (int kk = 1; kk < 4; ++kk)
+                            ptx::mma_ss_c<true>(tmem_O, ptx::make_desc(p_lo + kk * 2, kDescHiK),
+                                                ptx::make_desc(v_lo + kk * (2048 >> 4), kDescHiK), kIdescPV);
+                        // the P buffer may be overwritten (and O_t rescaled) once these MMAs have retired
+                        ptx::tc_commit(b_pfree);
+                    }
+                    if (!ok) break;
                     first_pv = false;
-                    kv_release(stage);
+                    ++n_pv;
+                    kv_release(stage_v);
                     if (!has_next) {
                         ptx::tc_commit(ptx::smem_u32(&ctrl->o_full[t]));
                         break;
                     }
-                    issue_qk(nxt);
+                    if (!qk_done) issue_qk(nxt, kNone);
                     cur = nxt;
                     s = s2;
                 }
                 ++n_it;
                 ring_base += (uint32_t)item.n_loads;
-                kv_pass_until(ring_base);
+                kv_walk(ring_base, kNone);
             }
             if (*abort_flag) {
                 // MMAs that were issued must retire before tensor memory is given back
@@ -475,7 +528,10 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         const float c = prm.scale_log2;
         // the table of Eq. 3's half widths: shared memory when it fits, else global memory
         const int32_t *half_width = prm.n_half_width <= kHalfWidthSmem ? ctrl->half_width : prm.half_width;
-        const uint32_t b_s = ptx::smem_u32(&ctrl->s_full[t]), b_p = ptx::smem_u32(&ctrl->p_ready[t]);
+        const uint32_t b_s = ptx::smem_u32(&ctrl->s_full[t]), b_sfree = ptx::smem_u32(&ctrl->s_free[t]);
+        const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]);
+        // this row of the P half-tile: K-major, 128-byte rows, 16-byte chunks XOR-swizzled by the row number
+        uint8_t *p_row = smem_raw + (sP - smem_base) + t * kHalfBytes + r * 128;
         uint32_t n_s = 0, n_items_seen = 0;
         bool alive = true;
         for (uint32_t k = 0; alive; ++k) {
@@ -578,32 +634,23 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
 #pragma unroll
                 for (int w = 0; w < 4; ++w) ptx::tmem_ld32(tmem_S + lane_off + 32 * w, sv[w]);
                 ptx::tmem_wait_ld();
+                // S_t is in registers: the next Q_t K^T may overwrite it
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(b_sfree);
 
-                // Groups of 16 keys (one grid row of a key patch) that no query of this warp may see are
-                // skipped altogether: bit g of `live` = some lane has an allowed key in group g.
-                uint32_t live = 0xffu;
-                if (masked) {
-                    live = 0u;
-#pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        if (__any_sync(0xffffffffu, ((mw[g >> 1] >> (16 * (g & 1))) & 0xffffu) != 0u)) live |= 1u << g;
-                }
                 // row maximum over the allowed keys, four independent chains of three-input maxima
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 if (masked) {
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        if (!(live & (1u << g))) continue;
-                        const int w = g >> 1;
+                    for (int w = 0; w < 4; ++w)
 #pragma unroll
-                        for (int j = 16 * (g & 1); j < 16 * (g & 1) + 16; j += 2) {
+                        for (int j = 0; j < 32; j += 2) {
                             const float v0 = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
                             const float v1 = ((mw[w] >> (j + 1)) & 1u) ? __uint_as_float(sv[w][j + 1]) : -INFINITY;
                             sv[w][j] = __float_as_uint(v0);
                             sv[w][j + 1] = __float_as_uint(v1);
                             mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], v0, v1);
                         }
-                    }
                 } else {
 #pragma unroll
                     for (int w = 0; w < 4; ++w)
@@ -613,6 +660,15 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 }
                 const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
 
+                // Every P_t V issued so far must have retired before O_t is rescaled or the P buffer is
+                // written again (completion 2 i - 1 of the barrier: second half of the previous step).
+                if (n_s > 1) {
+                    if (!__all_sync(0xffffffffu, wait_bar(b_pfree, 1u, abort_flag, prm.status, 17))) {
+                        alive = false;
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                }
                 // ---- running maximum; O is rescaled only when it grew by more than the threshold -----
                 const float m_new = fmaxf(m_used, mx);
                 if (first) {
@@ -646,37 +702,46 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 const uint64_t c2 = ptx::pack2(c, c), nmc2 = ptx::pack2(-mc, -mc);
                 uint64_t lsum[2] = {0ull, 0ull};
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        if (live & (1u << (2 * w + hh))) {
-#pragma unroll
-                            for (int j = 16 * hh; j < 16 * hh + 16; j += 2) {
-                                const uint64_t x2 =
-                                    ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
-                                float x0, x1;
-                                ptx::unpack2(x2, x0, x1);
-                                const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
-                                lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
-                                pk[j >> 1] = ptx::pack_bf16(p0, p1);
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 8 * hh; j < 8 * hh + 8; ++j) pk[j] = 0u;
+                for (int h = 0; h < 2; ++h) {
+                    if (h == 1) {
+                        // the first half's P_t V must have read the buffer (completion 2 i of the barrier)
+                        if (!__all_sync(0xffffffffu, wait_bar(b_pfree, 0u, abort_flag, prm.status, 18))) {
+                            alive = false;
+                            break;
                         }
                     }
-                    ptx::tmem_st16(tmem_S + lane_off + 16 * w, pk);
+#pragma unroll
+                    for (int gg = 0; gg < 4; ++gg) {
+                        const int g = 4 * h + gg, w = g >> 1;  // group of 16 keys: chunks 2 gg and 2 gg + 1 of the row
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int j = 16 * (g & 1); j < 16 * (g & 1) + 16; j += 2) {
+                            const uint64_t x2 =
+                                ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
+                            float x0, x1;
+                            ptx::unpack2(x2, x0, x1);
+                            const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
+                            lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
+                            pk[(j >> 1) & 7] = ptx::pack_bf16(p0, p1);
+                        }
+#pragma unroll
+                        for (int cc = 0; cc < 2; ++cc) {
+                            const int ch = 2 * gg + cc;
+                            *reinterpret_cast<uint4 *>(p_row + ((ch ^ (r & 7)) << 4)) =
+                                make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+                        }
+                    }
+                    // generic-proxy writes -> visible to the tensor core's (async proxy) reads
+                    ptx::fence_proxy_async_smem();
+                    ptx::mbar_arrive(ptx::smem_u32(&ctrl->p_ready[t][h]));
                 }
+                if (!alive) break;
                 {
                     float a0, a1, a2, a3;
                     ptx::unpack2(lsum[0], a0, a1);
                     ptx::unpack2(lsum[1], a2, a3);
                     l += (a0 + a1) + (a2 + a3);
                 }
-                ptx::tmem_wait_st();
-                ptx::tc_fence_before();
-                ptx::mbar_arrive(b_p);
             }
             if (!alive) break;
 
@@ -874,7 +939,7 @@ std::mutex g_dev_mutex;
 template <int D>
 int launch_variant(const clear_plan &p, const CUtensorMap *tm, const WsParams &prm, cudaStream_t stream)
 {
-    constexpr size_t kSmem = (size_t)(2 + kRing) * (D / 64) * 16384 + sizeof(Ctrl);
+    constexpr size_t kSmem = (size_t)(2 + kRing) * (D / 64) * 16384 + 2 * 16384 + sizeof(Ctrl);
     static_assert(kSmem <= 232448, "shared memory of one block");
     int n_sm = 0;
     {
