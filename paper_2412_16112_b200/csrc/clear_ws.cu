@@ -78,14 +78,19 @@ struct Ctrl {
     int32_t half_width[kHalfWidthSmem];
 };
 
-// Bounded wait on an mbarrier phase.  Returns false once the block has given up.  A waiting thread
-// sleeps inside try_wait (suspend-time hint) rather than spinning: a spinning warp would take issue
-// slots and instruction-cache lines from the softmax warps of its scheduler.
+// Bounded wait on an mbarrier phase.  Returns false once the block has given up.  The polling loop is
+// kept to two instructions per try, and roles that can afford it (SLEEP_NS > 0) sleep between tries:
+// a busily polling warp takes issue slots and instruction-cache lines from the softmax warps.
+template <uint32_t SLEEP_NS>
 __device__ __forceinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
 {
     const uint64_t t0 = ptx::globaltimer_ns();
     for (;;) {
-        if (ptx::mbar_try_wait_hint(bar, parity, kWaitHintNs)) return true;
+#pragma unroll 1
+        for (int i = 0; i < 128; ++i) {
+            if (ptx::mbar_try_wait_hint(bar, parity, kWaitHintNs)) return true;
+            if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+        }
         if (*abort_flag) return false;
         if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) break;
     }
@@ -93,10 +98,17 @@ __device__ __forceinline__ bool wait_bar_slow(uint32_t bar, uint32_t parity, vol
     atomicCAS(status, 0, code);  // the first wait that expired names the cause
     return false;
 }
+template <uint32_t SLEEP_NS = 0>
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status, int code)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
-    return wait_bar_slow(bar, parity, abort_flag, status, code);
+    return wait_bar_slow<SLEEP_NS>(bar, parity, abort_flag, status, code);
+}
+// One arrival for the whole warp, after every lane has got here (and its earlier writes with it).
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
+{
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(bar);
 }
 // Drain: wait for a phase regardless of the abort flag (used before leaving with copies in flight).
 __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity)
@@ -233,14 +245,14 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_empty[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->s_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->s_free[i]), 128);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][0]), 128);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][1]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->s_free[i]), 4);  // one arrival per warp
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][0]), 4);  // one arrival per warp
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][1]), 4);  // one arrival per warp
             ptx::mbar_init(ptx::smem_u32(&ctrl->p_free[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->o_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 128);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->stats_full[i]), 128);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->stats_empty[i]), 128);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 4);  // one arrival per warp
+            ptx::mbar_init(ptx::smem_u32(&ctrl->stats_full[i]), 4);  // one arrival per warp
+            ptx::mbar_init(ptx::smem_u32(&ctrl->stats_empty[i]), 4);  // one arrival per warp
         }
         for (int i = 0; i < kRing; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->kv_full[i]), 1);
@@ -272,7 +284,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             uint32_t n_q[2] = {0, 0};
             for (uint32_t k = 0;; ++k) {
                 const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
-                if (!wait_bar(ptx::smem_u32(&ctrl->sched_empty[slot]), (use & 1u) ^ 1u, abort_flag, prm.status, 1)) break;
+                if (!wait_bar<200>(ptx::smem_u32(&ctrl->sched_empty[slot]), (use & 1u) ^ 1u, abort_flag, prm.status, 1)) break;
                 const int g = atomicAdd(prm.status + 1, 1);
                 ItemRef ref{0, 0};
                 clear_pair_item_t item{};
@@ -288,7 +300,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 bool ok = true;
                 for (int t = 0; t < item.n_sides && ok; ++t) {
                     const uint32_t bar = ptx::smem_u32(&ctrl->q_full[t]);
-                    ok = wait_bar(ptx::smem_u32(&ctrl->q_empty[t]), (n_q[t] & 1u) ^ 1u, abort_flag, prm.status, 2);
+                    ok = wait_bar<200>(ptx::smem_u32(&ctrl->q_empty[t]), (n_q[t] & 1u) ^ 1u, abort_flag, prm.status, 2);
                     if (!ok) break;
                     ptx::mbar_expect_tx(bar, kTileBytes);
 #pragma unroll
@@ -316,7 +328,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         for (int t = 0; t < 2; ++t) {
                             if (!ok || (t == 0 ? !has_a : !has_b)) continue;
                             const uint32_t stage = n_loads % kRing, fill = n_loads / kRing;
-                            ok = wait_bar(ptx::smem_u32(&ctrl->kv_empty[stage]), (fill & 1u) ^ 1u, abort_flag, prm.status, 3);
+                            ok = wait_bar<100>(ptx::smem_u32(&ctrl->kv_empty[stage]), (fill & 1u) ^ 1u, abort_flag, prm.status, 3);
                             if (!ok) continue;
                             const uint32_t bar = ptx::smem_u32(&ctrl->kv_full[stage]);
                             const uint32_t dst = sRing + stage * kTileBytes;
@@ -636,7 +648,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 ptx::tmem_wait_ld();
                 // S_t is in registers: the next Q_t K^T may overwrite it
                 ptx::tc_fence_before();
-                ptx::mbar_arrive(b_sfree);
+                warp_arrive(b_sfree, lane);
 
                 // row maximum over the allowed keys, four independent chains of three-input maxima
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -703,6 +715,22 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 uint64_t lsum[2] = {0ull, 0ull};
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
+                    // this half of the row (64 keys) as 32 bf16 pairs, kept in registers until the buffer is free
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int w2 = 0; w2 < 2; ++w2) {
+                        const int w = 2 * h + w2;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            const uint64_t x2 =
+                                ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
+                            float x0, x1;
+                            ptx::unpack2(x2, x0, x1);
+                            const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
+                            lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
+                            pk[16 * w2 + (j >> 1)] = ptx::pack_bf16(p0, p1);
+                        }
+                    }
                     if (h == 1) {
                         // the first half's P_t V must have read the buffer (completion 2 i of the barrier)
                         if (!__all_sync(0xffffffffu, wait_bar(b_pfree, 0u, abort_flag, prm.status, 18))) {
@@ -711,29 +739,12 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         }
                     }
 #pragma unroll
-                    for (int gg = 0; gg < 4; ++gg) {
-                        const int g = 4 * h + gg, w = g >> 1;  // group of 16 keys: chunks 2 gg and 2 gg + 1 of the row
-                        uint32_t pk[8];
-#pragma unroll
-                        for (int j = 16 * (g & 1); j < 16 * (g & 1) + 16; j += 2) {
-                            const uint64_t x2 =
-                                ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
-                            float x0, x1;
-                            ptx::unpack2(x2, x0, x1);
-                            const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
-                            lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
-                            pk[(j >> 1) & 7] = ptx::pack_bf16(p0, p1);
-                        }
-#pragma unroll
-                        for (int cc = 0; cc < 2; ++cc) {
-                            const int ch = 2 * gg + cc;
-                            *reinterpret_cast<uint4 *>(p_row + ((ch ^ (r & 7)) << 4)) =
-                                make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-                        }
-                    }
+                    for (int ch = 0; ch < 8; ++ch)
+                        *reinterpret_cast<uint4 *>(p_row + ((ch ^ (r & 7)) << 4)) =
+                            make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
                     // generic-proxy writes -> visible to the tensor core's (async proxy) reads
                     ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(ptx::smem_u32(&ctrl->p_ready[t][h]));
+                    warp_arrive(ptx::smem_u32(&ctrl->p_ready[t][h]), lane);
                 }
                 if (!alive) break;
                 {
@@ -750,7 +761,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                                                   prm.status, 11)))
                 break;
             ctrl->stats[t][r] = make_float2(m_used * c, l);
-            ptx::mbar_arrive(ptx::smem_u32(&ctrl->stats_full[t]));
+            warp_arrive(ptx::smem_u32(&ctrl->stats_full[t]), lane);
             ++n_items_seen;
         }
     } else {
@@ -762,7 +773,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         bool alive = true;
         for (uint32_t k = 0; alive; ++k) {
             const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
-            if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 12)))
+            if (!__all_sync(0xffffffffu, wait_bar<500>(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 12)))
                 break;
             const int g = ctrl->sched_item[slot];
             const clear_pair_item_t item = ctrl->sched_rec[slot];
@@ -773,13 +784,13 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             if (g >= total_items) break;
             for (int t = 0; t < item.n_sides; ++t) {
                 const uint32_t ph = n_seen[t] & 1u;
-                if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->stats_full[t]), ph, abort_flag, prm.status, 13))) {
+                if (!__all_sync(0xffffffffu, wait_bar<500>(ptx::smem_u32(&ctrl->stats_full[t]), ph, abort_flag, prm.status, 13))) {
                     alive = false;
                     break;
                 }
                 const float2 ml = ctrl->stats[t][r];
-                ptx::mbar_arrive(ptx::smem_u32(&ctrl->stats_empty[t]));
-                if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->o_full[t]), ph, abort_flag, prm.status, 14))) {
+                warp_arrive(ptx::smem_u32(&ctrl->stats_empty[t]), lane);
+                if (!__all_sync(0xffffffffu, wait_bar<200>(ptx::smem_u32(&ctrl->o_full[t]), ph, abort_flag, prm.status, 14))) {
                     alive = false;
                     break;
                 }
@@ -809,7 +820,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         ptx::tmem_wait_ld();
                         if (w == D / 32 - 1) {
                             ptx::tc_fence_before();
-                            ptx::mbar_arrive(ptx::smem_u32(&ctrl->o_empty[t]));
+                            warp_arrive(ptx::smem_u32(&ctrl->o_empty[t]), lane);
                         }
                         if (q_valid) {
 #pragma unroll
@@ -831,7 +842,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         ptx::tmem_wait_ld();
                         if (w == D / 32 - 1) {
                             ptx::tc_fence_before();
-                            ptx::mbar_arrive(ptx::smem_u32(&ctrl->o_empty[t]));
+                            warp_arrive(ptx::smem_u32(&ctrl->o_empty[t]), lane);
                         }
                         if (q_valid) {
 #pragma unroll
