@@ -238,16 +238,28 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
     };
 
     auto finish_item = [&](clear_pair_item_t &it) {
-        int32_t loads = 0;
-        for (int32_t i = it.step_begin; i < (int32_t)sch.pair_steps.size(); ++i) {
-            clear_pair_step_t &st = sch.pair_steps[(size_t)i];
-            st.load_base = loads;
+        // staging order: K(0), then K(s + 1), V(s) for every step s (K runs one step ahead of V)
+        auto n_tiles = [&](int32_t i) {
+            const clear_pair_step_t &st = sch.pair_steps[(size_t)i];
             const int a = (st.flags & CLEAR_STEP_USE0) ? 1 : 0;
             const int b = ((st.flags & CLEAR_STEP_USE1) && !(st.flags & CLEAR_STEP_SHARED)) ? 1 : 0;
-            loads += 2 * (a + b);
+            return a + b;
+        };
+        const int32_t first = it.step_begin, end = (int32_t)sch.pair_steps.size();
+        int32_t pos = 0;
+        std::vector<int32_t> k_pos((size_t)(end - first), 0);
+        k_pos[0] = pos;
+        pos += n_tiles(first);
+        for (int32_t i = first; i < end; ++i) {
+            if (i + 1 < end) {
+                k_pos[(size_t)(i + 1 - first)] = pos;
+                pos += n_tiles(i + 1);
+            }
+            sch.pair_steps[(size_t)i].load_base = k_pos[(size_t)(i - first)] | (pos << 16);
+            pos += n_tiles(i);
         }
-        it.step_count = (int32_t)sch.pair_steps.size() - it.step_begin;
-        it.n_loads = loads;
+        it.step_count = end - first;
+        it.n_loads = pos;
         sch.pair_items.push_back(it);
     };
     auto linear_step = [&](int x, int n_valid, int n_sides) {

@@ -5,19 +5,20 @@
 // text tokens -- and a list of steps; in each step every query tile of the pair meets one 128-key
 // tile (Eq. 1 restricted by Eq. 3).  Key tiles both query tiles need are staged once.
 //
-// Roles (512 threads):
+// Roles (640 threads):
 //   warp 0        : takes items from the queue and issues every TMA load (Q tiles, K/V ring);
 //   warps 1, 2    : one thread each issues the tcgen05.mma of query tile t = 0, 1: S_t = Q_t K^T,
 //                   O_t += P_t V; the softmax of one query tile runs under the MMAs of the other;
-//   warps 4-7     : softmax of query tile 0 (thread r owns query row r = tensor-memory lane r):
-//                   mask, running maximum, P = exp2(.), row sum, P (bf16) back into tensor memory;
-//   warps 8-11    : the same for query tile 1;
-//   warps 12-15   : epilogue: O / l -> bf16 -> global memory (or fp32 partial results of split
-//                   text rows), while the other warps already run the next item.
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each.  P goes through shared memory, 64
-// keys at a time, so that S_t of the next step can be computed while the softmax of this one runs.
-// Shared memory: Q0, Q1, a ring of four key/value stages (K and V tiles take one stage each) and one
-// half-tile of P per query tile.
+//   warps 4-11    : softmax and epilogue of query tile 0, two threads per query row (= tensor-memory
+//                   lane), each with half of the keys of every tile: mask, maximum, P = exp2(.) as bf16
+//                   into shared memory, row sum; at the end of an item O / l -> bf16 -> global memory
+//                   (or fp32 partial results of split text rows);
+//   warps 12-19   : the same for query tile 1.
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each.  P goes through shared memory, so
+// that S_t of the next step can be computed while the softmax of this one runs; it is handed to the
+// tensor core 64 keys at a time.
+// Shared memory: Q0, Q1, a ring of three key/value stages (K and V tiles take one stage each) and P
+// of each query tile.
 // Every wait is bounded: on expiry the block raises the plan's status word and leaves.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -31,19 +32,19 @@
 namespace clear {
 namespace {
 
-constexpr int kWsThreads = 512;
-constexpr int kRing = 4;
+constexpr int kWsThreads = 640;   // 4 control warps + 2 x 8 softmax warps
+constexpr int kRing = 3;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr uint32_t kWaitHintNs = 20000;            // one sleep inside try_wait
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the row max grows by more
 constexpr int kSchedDepth = 2;
-// arrivals that free a queue slot: the two MMA threads and one lane of each of the 12 softmax / epilogue warps
-constexpr uint32_t kSchedReaders = 14;
-// registers per thread of each role (warpgroups of 128 threads: 72 + 2 * 184 + 72 = 512)
-constexpr uint32_t kRegsControl = 72, kRegsSoftmax = 184, kRegsEpilogue = 72;
-constexpr int kHalfWidthSmem = 128;  // entries of the half-width table kept in shared memory
+// arrivals that free a queue slot: the two MMA threads and one lane of each of the 16 softmax warps
+constexpr uint32_t kSchedReaders = 18;
+// registers per thread of each role: 128 x 64 + 512 x 104 = 61440 = what the block is launched with
+// (640 threads x 96); raising a warp's budget only draws on registers other warps of the block gave back
+constexpr uint32_t kRegsControl = 64, kRegsSoftmax = 104;
 
 struct WsParams {
     const clear_pair_item_t *items;
@@ -65,7 +66,8 @@ struct WsParams {
 struct Ctrl {
     uint64_t q_full[2], q_empty[2];
     uint64_t kv_full[kRing], kv_empty[kRing];
-    uint64_t s_full[2], s_free[2], p_ready[2][2], p_free[2], o_full[2], o_empty[2], stats_full[2], stats_empty[2];
+    uint64_t s_full[2], s_free[2], p_ready[2][2], p_free[2], o_full[2], o_empty[2];
+    uint64_t pair[2][4];  // the two warps that share 32 query rows of a tile
     uint64_t sched_full[kSchedDepth], sched_empty[kSchedDepth];
     uint64_t drain[2];
     int32_t sched_item[kSchedDepth];            // queue position, >= total: no more work
@@ -74,8 +76,9 @@ struct Ctrl {
     uint32_t tmem_base;
     int abort_flag;
     int skip;
-    float2 stats[2][128];  // per query row: running maximum (log2 units) and row sum
-    int32_t half_width[kHalfWidthSmem];
+    // [query tile][slot][thread of the row][row]: the row maxima (16 bits each) the two threads of a row
+    // show each other, two slots used in turn; at the end of an item each slot holds 128 fp32 row sums
+    alignas(16) uint16_t xchg[2][2][2][128];
 };
 
 // Bounded wait on an mbarrier phase.  Returns false once the block has given up.  The polling loop is
@@ -160,32 +163,28 @@ __device__ __forceinline__ clear_pair_item_t load_item(const clear_pair_item_t *
     it.step_count = c.x; it.n_loads = c.y; it.partial_slot0 = c.z; it.partial_slot1 = c.w;
     return it;
 }
-// The part of a step record one query tile of the pair needs.
+// The part of a step record the softmax of one query tile of the pair needs on every step.
 struct SideStep {
-    int x, y, flags, n_valid;
+    int flags, n_valid;
 };
 __device__ __forceinline__ SideStep load_side_step(const clear_pair_step_t *p, int side)
 {
-    const int4 a = __ldg(reinterpret_cast<const int4 *>(p));
     const int4 b = __ldg(reinterpret_cast<const int4 *>(p) + 1);
     SideStep s;
-    s.x = side ? a.z : a.x;
-    s.y = side ? a.w : a.y;
     s.flags = b.x;
     s.n_valid = side ? b.z : b.y;
     return s;
 }
+// Origin of the key patch of that tile (only clipped patches and plans without a mask table need it).
+__device__ __forceinline__ int2 load_side_origin(const clear_pair_step_t *p, int side)
+{
+    const int4 a = __ldg(reinterpret_cast<const int4 *>(p));
+    return side ? make_int2(a.z, a.w) : make_int2(a.x, a.y);
+}
 static_assert(sizeof(clear_pair_step_t) == 32 && sizeof(clear_pair_item_t) == 48, "table records are read as int4");
 
 __device__ __forceinline__ bool step_uses(int flags, int side) { return (flags & (side ? CLEAR_STEP_USE1 : CLEAR_STEP_USE0)) != 0; }
-// Ring positions (relative to the step's load_base) of the K and V tiles a side reads in a step:
-// stages are filled in the order K(tile 0), K(tile 1), V(tile 0), V(tile 1), skipping what is absent.
-__device__ __forceinline__ int step_n_tiles(int flags)
-{
-    const int a = (flags & CLEAR_STEP_USE0) ? 1 : 0;
-    const int b = ((flags & CLEAR_STEP_USE1) && !(flags & CLEAR_STEP_SHARED)) ? 1 : 0;
-    return a + b;
-}
+// A step's K tiles, and its V tiles, take one ring position per distinct key tile (tile 0's first):
 __device__ __forceinline__ int step_tile_index(int flags, int side)
 {
     if (side == 0 || (flags & CLEAR_STEP_SHARED)) return 0;
@@ -207,9 +206,9 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t smem_base = ptx::smem_u32(smem_raw);
-    // Q0, Q1 | ring of K/V stages | one half-tile of P (128 queries x 64 keys) per query tile | control
+    // Q0, Q1 | ring of K/V stages | P of each query tile as two half-tiles (128 queries x 64 keys) | control
     const uint32_t sQ = smem_base, sRing = sQ + 2 * kTileBytes, sP = sRing + kRing * kTileBytes;
-    constexpr uint32_t kCtrlOff = (2 + kRing) * kTileBytes + 2 * kHalfBytes;
+    constexpr uint32_t kCtrlOff = (2 + kRing) * kTileBytes + 4 * kHalfBytes;
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_raw + kCtrlOff);
     volatile int *abort_flag = &ctrl->abort_flag;
 
@@ -245,14 +244,13 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_empty[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->s_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->s_free[i]), 4);  // one arrival per warp
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][0]), 4);  // one arrival per warp
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][1]), 4);  // one arrival per warp
+            ptx::mbar_init(ptx::smem_u32(&ctrl->s_free[i]), 8);  // one arrival per softmax warp of the tile
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][0]), 8);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][1]), 8);
             ptx::mbar_init(ptx::smem_u32(&ctrl->p_free[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->o_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 4);  // one arrival per warp
-            ptx::mbar_init(ptx::smem_u32(&ctrl->stats_full[i]), 4);  // one arrival per warp
-            ptx::mbar_init(ptx::smem_u32(&ctrl->stats_empty[i]), 4);  // one arrival per warp
+            ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 8);
+            for (int j = 0; j < 4; ++j) ptx::mbar_init(ptx::smem_u32(&ctrl->pair[i][j]), 2);
         }
         for (int i = 0; i < kRing; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->kv_full[i]), 1);
@@ -266,7 +264,6 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         ptx::mbar_init(ptx::smem_u32(&ctrl->drain[1]), 1);
         ptx::fence_mbar_init();
     }
-    for (int i = tid; i < prm.n_half_width && i < kHalfWidthSmem; i += kWsThreads) ctrl->half_width[i] = prm.half_width[i];
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), kTmemCols);
         ptx::tmem_relinquish();
@@ -313,37 +310,45 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     }
                     ++n_q[t];
                 }
-                const clear_pair_step_t *steps = prm.steps + item.step_begin;
-                clear_pair_step_t st_next = load_step(steps);
-                for (int s = 0; s < item.step_count && ok; ++s) {
-                    // the next record is fetched one step ahead, so its latency is off the critical path
-                    const clear_pair_step_t st = st_next;
-                    if (s + 1 < item.step_count) st_next = load_step(steps + s + 1);
+                // K/V stages in the plan's staging order: K(step 0), then K(step s + 1), V(step s) for every
+                // step s, so that a step's K tile is on its way a whole step before its V tile is needed
+                auto stage_tiles = [&](const clear_pair_step_t &st, int kv) {
                     const bool has_a = (st.flags & CLEAR_STEP_USE0) != 0;
                     const bool has_b = (st.flags & CLEAR_STEP_USE1) && !(st.flags & CLEAR_STEP_SHARED);
                     const bool linear = (st.flags & CLEAR_STEP_LINEAR) != 0;
 #pragma unroll
-                    for (int kv = 0; kv < 2; ++kv) {
+                    for (int t = 0; t < 2; ++t) {
+                        if (!ok || (t == 0 ? !has_a : !has_b)) continue;
+                        const uint32_t stage = n_loads % kRing, fill = n_loads / kRing;
+                        ok = wait_bar<100>(ptx::smem_u32(&ctrl->kv_empty[stage]), (fill & 1u) ^ 1u, abort_flag, prm.status, 3);
+                        if (!ok) continue;
+                        const uint32_t bar = ptx::smem_u32(&ctrl->kv_full[stage]);
+                        const uint32_t dst = sRing + stage * kTileBytes;
+                        const int x = t ? st.x1 : st.x0, y = t ? st.y1 : st.y0;
+                        ptx::mbar_expect_tx(bar, kTileBytes);
 #pragma unroll
-                        for (int t = 0; t < 2; ++t) {
-                            if (!ok || (t == 0 ? !has_a : !has_b)) continue;
-                            const uint32_t stage = n_loads % kRing, fill = n_loads / kRing;
-                            ok = wait_bar<100>(ptx::smem_u32(&ctrl->kv_empty[stage]), (fill & 1u) ^ 1u, abort_flag, prm.status, 3);
-                            if (!ok) continue;
-                            const uint32_t bar = ptx::smem_u32(&ctrl->kv_full[stage]);
-                            const uint32_t dst = sRing + stage * kTileBytes;
-                            const int x = t ? st.x1 : st.x0, y = t ? st.y1 : st.y0;
-                            ptx::mbar_expect_tx(bar, kTileBytes);
-#pragma unroll
-                            for (int h = 0; h < kHalves; ++h) {
-                                if (linear)
-                                    ptx::tma_load_3d(dst + h * kHalfBytes, kv ? &tm_v_lin : &tm_k_lin, bar, h * 64, x, ref.bh);
-                                else
-                                    ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_v_img : &tm_k_img, bar, h * 64, x, y, ref.bh);
-                            }
-                            ++n_loads;
+                        for (int h = 0; h < kHalves; ++h) {
+                            if (linear)
+                                ptx::tma_load_3d(dst + h * kHalfBytes, kv ? &tm_v_lin : &tm_k_lin, bar, h * 64, x, ref.bh);
+                            else
+                                ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_v_img : &tm_k_img, bar, h * 64, x, y, ref.bh);
                         }
+                        ++n_loads;
                     }
+                };
+                const clear_pair_step_t *steps = prm.steps + item.step_begin;
+                clear_pair_step_t st = load_step(steps);
+                clear_pair_step_t st_next = st;
+                if (item.step_count > 1) st_next = load_step(steps + 1);
+                stage_tiles(st, 0);
+                for (int s = 0; s < item.step_count && ok; ++s) {
+                    // records are fetched ahead of their use, so their latency is off the critical path
+                    clear_pair_step_t st_next2 = st_next;
+                    if (s + 2 < item.step_count) st_next2 = load_step(steps + s + 2);
+                    if (s + 1 < item.step_count) stage_tiles(st_next, 0);
+                    stage_tiles(st, 1);
+                    st = st_next;
+                    st_next = st_next2;
                 }
                 if (!ok) break;
             }
@@ -365,7 +370,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             const int t = warp - 1;
             constexpr uint32_t kDescHiK = ptx::smem_desc_hi_sw128(1024);  // 8-row groups are 1024 bytes apart
             const uint32_t q_lo = ptx::smem_desc_lo(sQ + t * kTileBytes, 16);
-            const uint32_t p_lo = ptx::smem_desc_lo(sP + t * kHalfBytes, 16);
+            const uint32_t p_lo = ptx::smem_desc_lo(sP + t * 2 * kHalfBytes, 16);
             const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
             const uint32_t b_sfull = ptx::smem_u32(&ctrl->s_full[t]), b_sfree = ptx::smem_u32(&ctrl->s_free[t]);
             const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]);
@@ -423,7 +428,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     // the softmax warps must have taken the previous S_t out of tensor memory
                     if (n_qk > 0) ok = wait_bar(b_sfree, (n_qk - 1) & 1u, abort_flag, prm.status, 16);
                     if (!ok) return;
-                    const uint32_t pos = ring_base + (uint32_t)st.load_base + (uint32_t)step_tile_index(st.flags, t);
+                    const uint32_t pos = ring_base + ((uint32_t)st.load_base & 0xffffu) + (uint32_t)step_tile_index(st.flags, t);
                     const uint32_t stage = kv_wait(pos, keep);
                     if (!ok) return;
                     ptx::tc_fence_after();
@@ -440,8 +445,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     ++n_qk;
                 };
                 auto v_position = [&](const clear_pair_step_t &st) -> uint32_t {
-                    return ring_base + (uint32_t)st.load_base + (uint32_t)step_n_tiles(st.flags) +
-                           (uint32_t)step_tile_index(st.flags, t);
+                    return ring_base + ((uint32_t)st.load_base >> 16) + (uint32_t)step_tile_index(st.flags, t);
                 };
 
                 // first step this query tile takes part in (every tile has at least one)
@@ -466,13 +470,14 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     if (!has_next) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
 
                     const uint32_t pos_v = v_position(cur);
-                    // The next S_t goes ahead of this step's P_t V when its K tile sits right behind this V
-                    // tile in the ring; a V tile held back for longer would stall the ring.
+                    // The next S_t goes ahead of this step's P_t V whenever its K tile was staged before this
+                    // step's V tile (it is, unless this query tile sits out the steps in between): the ring
+                    // is walked in staging order.
                     bool qk_done = false;
                     if (has_next) {
-                        const uint32_t pos_k = ring_base + (uint32_t)nxt.load_base + (uint32_t)step_tile_index(nxt.flags, t);
-                        if (pos_k - pos_v <= 2u) {
-                            issue_qk(nxt, pos_v);
+                        const uint32_t pos_k = ring_base + ((uint32_t)nxt.load_base & 0xffffu) + (uint32_t)step_tile_index(nxt.flags, t);
+                        if (pos_k < pos_v) {
+                            issue_qk(nxt, kNone);
                             qk_done = true;
                             if (!ok) break;
                         }
@@ -498,14 +503,15 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         // P half: K-major, 16 keys are 32 bytes along a row; V: MN-major, 16 keys are 16
                         // rows of 128 bytes = 2048 bytes
                         const uint32_t v_lo = ptx::smem_desc_lo(sRing + stage_v * kTileBytes, kHalfBytes) + h * 4 * (2048 >> 4);
-                        ptx::mma_ss(tmem_O, ptx::make_desc(p_lo, kDescHiK), ptx::make_desc(v_lo, kDescHiK), kIdescPV,
+                        const uint32_t ph_lo = p_lo + h * (kHalfBytes >> 4);
+                        ptx::mma_ss(tmem_O, ptx::make_desc(ph_lo, kDescHiK), ptx::make_desc(v_lo, kDescHiK), kIdescPV,
                                     (first_pv && h == 0) ? 0u : 1u);
 #pragma unroll
                         for (int kk = 1; kk < 4; ++kk)
-                            ptx::mma_ss_c<true>(tmem_O, ptx::make_desc(p_lo + kk * 2, kDescHiK),
+                            ptx::mma_ss_c<true>(tmem_O, ptx::make_desc(ph_lo + kk * 2, kDescHiK),
                                                 ptx::make_desc(v_lo + kk * (2048 >> 4), kDescHiK), kIdescPV);
-                        // the P buffer may be overwritten (and O_t rescaled) once these MMAs have retired
-                        ptx::tc_commit(b_pfree);
+                        // P may be overwritten (and O_t rescaled) once this step's MMAs have retired
+                        if (h == 1) ptx::tc_commit(b_pfree);
                     }
                     if (!ok) break;
                     first_pv = false;
@@ -530,107 +536,131 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             }
         }
         __syncwarp();
-    } else if (warp < 12) {
-        // ================= softmax warps: thread r owns query row r of its tile =========================
+    } else {
+        // ================= softmax warps ===================================================================
+        // Eight warps per query tile, two threads per query row (tensor-memory lane): the thread with
+        // hf = 0 takes keys [0, 32) and [64, 96) of every 128-key tile, its partner (hf = 1, four warps
+        // further on) keys [32, 64) and [96, 128).  Four such warps per scheduler hide each other's
+        // instruction latencies.  The two threads of a row agree on the row maximum through shared
+        // memory once per tile and add up their row sums once per item; each normalises and stores half
+        // of the output channels.
         ptx::setmaxnreg_inc<kRegsSoftmax>();
-        const int t = (warp - 4) >> 2;           // query tile of the pair
-        const int r = tid & 127;
-        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
+        const int ws = warp - 4;
+        const int t = ws >> 3;          // query tile of the pair
+        const int hf = (ws >> 2) & 1;
+        const int q4 = ws & 3;          // tensor-memory lane quadrant (= warp % 4)
+        const int r = q4 * 32 + lane;   // query row of the tile
+        constexpr int kChan = D / 2;    // output channels per thread
+        const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+        const uint32_t tmem_S = tmem + t * 128 + 32 * hf, tmem_O = tmem + 256 + t * 128 + kChan * hf;
         const float c = prm.scale_log2;
-        // the table of Eq. 3's half widths: shared memory when it fits, else global memory
-        const int32_t *half_width = prm.n_half_width <= kHalfWidthSmem ? ctrl->half_width : prm.half_width;
         const uint32_t b_s = ptx::smem_u32(&ctrl->s_full[t]), b_sfree = ptx::smem_u32(&ctrl->s_free[t]);
         const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]);
-        // this row of the P half-tile: K-major, 128-byte rows, 16-byte chunks XOR-swizzled by the row number
-        uint8_t *p_row = smem_raw + (sP - smem_base) + t * kHalfBytes + r * 128;
-        uint32_t n_s = 0, n_items_seen = 0;
+        const uint32_t b_pair = ptx::smem_u32(&ctrl->pair[t][q4]);
+        // this thread's 64 bytes of its row of the P half-tile: K-major, 128-byte rows, 16-byte chunks
+        // XOR-swizzled by the row number
+        uint8_t *p_row = smem_raw + (sP - smem_base) + t * 2 * kHalfBytes + r * 128;
+        uint32_t n_s = 0, n_pair = 0, n_items_seen = 0;
         bool alive = true;
+        // the two warps of a row meet: one arrival each, then both see what the other wrote before
+        auto pair_sync = [&]() -> bool {
+            warp_arrive(b_pair, lane);
+            const bool ok = __all_sync(0xffffffffu, wait_bar(b_pair, n_pair & 1u, abort_flag, prm.status, 19));
+            ++n_pair;
+            return ok;
+        };
         for (uint32_t k = 0; alive; ++k) {
             const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
             if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 9)))
                 break;
             const int g = ctrl->sched_item[slot];
-            const clear_pair_item_t item = ctrl->sched_rec[slot];
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
-            if (g >= total_items) break;
-            if (t >= item.n_sides) continue;
-            const clear_pair_step_t *steps = prm.steps + item.step_begin;
-            const bool is_text = item.kind == 1;
-            int q_y = 0, q_x = 0;
+            // The item's record stays in its queue slot until this warp is done with the item (the slot
+            // is given back at the end), so that only what every step needs lives in registers.
+            const volatile clear_pair_item_t *rec = &ctrl->sched_rec[slot];
+            if (g >= total_items || t >= rec->n_sides) {
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
+                if (g >= total_items) break;
+                continue;
+            }
+            const clear_pair_step_t *steps = prm.steps + rec->step_begin;
+            const int step_count = rec->step_count;
+            const bool is_text = rec->kind == 1;
+            // does this row's query exist?  (image tiles: its grid position lies on the grid)
             bool q_valid;
-            if (is_text) {
-                q_valid = r < (t ? item.n_rows1 : item.n_rows0);
-            } else {
-                q_y = (t ? item.qy1 : item.qy0) + (r >> 4);
-                q_x = item.qx + (r & 15);
-                q_valid = q_y < prm.grid_h && q_x < prm.grid_w;
+            {
+                const int q_y = (t ? rec->qy1 : rec->qy0) + (r >> 4), q_x = rec->qx + (r & 15);
+                q_valid = is_text ? r < (t ? rec->n_rows1 : rec->n_rows0) : (q_y < prm.grid_h && q_x < prm.grid_w);
             }
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
 
-            // Step records are fetched two steps ahead and this row's precomputed mask words one step
-            // ahead, so that neither latency is on the critical path.
+            // The next step's record is fetched at the top of a step and this row's precomputed mask words
+            // for it in the middle, so that neither latency is on the critical path.
             const int kMaskedBit = t ? CLEAR_STEP_MASKED1 : CLEAR_STEP_MASKED0;
-            auto load_mask_row = [&](const SideStep &q) -> uint4 {
-                if (step_uses(q.flags, t) && (q.flags & kMaskedBit) && !(q.flags & CLEAR_STEP_LINEAR) && q.n_valid >= 0)
-                    return __ldg(reinterpret_cast<const uint4 *>(prm.mask_table) + ((size_t)q.n_valid * 128 + r));
-                return make_uint4(0u, 0u, 0u, 0u);
+            auto load_mask_row = [&](const SideStep &q) -> uint2 {
+                if (step_uses(q.flags, t) && (q.flags & kMaskedBit) && !(q.flags & CLEAR_STEP_LINEAR) && q.n_valid >= 0) {
+                    const uint32_t *e = prm.mask_table + ((size_t)q.n_valid * 128 + r) * 4 + hf;
+                    return make_uint2(__ldg(e), __ldg(e + 2));
+                }
+                return make_uint2(0u, 0u);
             };
             SideStep st_next = load_side_step(steps, t);
-            SideStep st_next2 = st_next;
-            if (item.step_count > 1) st_next2 = load_side_step(steps + 1, t);
-            uint4 mrow_next = load_mask_row(st_next);
-            for (int s = 0; s < item.step_count; ++s) {
+            uint2 mrow_next = load_mask_row(st_next);
+            for (int s = 0; s < step_count; ++s) {
                 const SideStep st = st_next;
-                const uint4 mrow = mrow_next;
-                st_next = st_next2;
-                if (s + 2 < item.step_count) st_next2 = load_side_step(steps + s + 2, t);
-                if (s + 1 < item.step_count) mrow_next = load_mask_row(st_next);
-                if (!step_uses(st.flags, t)) continue;
+                const uint2 mrow = mrow_next;
+                if (s + 1 < step_count) st_next = load_side_step(steps + s + 1, t);
+                if (!step_uses(st.flags, t)) {
+                    if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
+                    continue;
+                }
                 const bool masked = (st.flags & kMaskedBit) != 0;
-                // ---- mask bits of this row for the tile (bit j = key j allowed) -----------------------
-                uint32_t mw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+                // ---- mask bits of this thread's keys: mw[i] bit j = key 64 i + 32 hf + j allowed -------
+                uint32_t mw[2] = {0xffffffffu, 0xffffffffu};
                 if (masked) {
                     if (st.flags & CLEAR_STEP_LINEAR) {
 #pragma unroll
-                        for (int w = 0; w < 4; ++w) {
-                            const int nv = min(max(st.n_valid - 32 * w, 0), 32);
-                            mw[w] = nv == 32 ? 0xffffffffu : ((1u << nv) - 1u);
+                        for (int i = 0; i < 2; ++i) {
+                            const int nv = min(max(st.n_valid - 32 * (2 * i + hf), 0), 32);
+                            mw[i] = nv == 32 ? 0xffffffffu : ((1u << nv) - 1u);
                         }
                     } else if (st.n_valid >= 0) {
                         // Eq. 3 from the table; keys of the patch that lie off the grid do not exist
                         mw[0] = mrow.x;
                         mw[1] = mrow.y;
-                        mw[2] = mrow.z;
-                        mw[3] = mrow.w;
                         if (st.flags & (t ? CLEAR_STEP_CLIP1 : CLEAR_STEP_CLIP0)) {
-                            const int lo = max(0, -st.x), hi = min(15, prm.grid_w - 1 - st.x);
+                            const int2 org = load_side_origin(steps + s, t);
+                            const int lo = max(0, -org.x), hi = min(15, prm.grid_w - 1 - org.x);
                             const uint32_t cols = lo <= hi ? (((1u << (hi - lo + 1)) - 1u) << lo) : 0u;
 #pragma unroll
-                            for (int w = 0; w < 4; ++w) {
-                                const int ky0 = st.y + 2 * w, ky1 = ky0 + 1;
+                            for (int i = 0; i < 2; ++i) {
+                                const int ky0 = org.y + 2 * (2 * i + hf), ky1 = ky0 + 1;
                                 const uint32_t ok0 = (ky0 >= 0 && ky0 < prm.grid_h) ? cols : 0u;
                                 const uint32_t ok1 = (ky1 >= 0 && ky1 < prm.grid_h) ? cols : 0u;
-                                mw[w] &= ok0 | (ok1 << 16);
+                                mw[i] &= ok0 | (ok1 << 16);
                             }
                         }
                     } else {
+                        // no table entry (very large radius): Eq. 3 row by row from the half widths
+                        const int2 org = load_side_origin(steps + s, t);
+                        const int q_y = (t ? rec->qy1 : rec->qy0) + (r >> 4), q_x = rec->qx + (r & 15);
 #pragma unroll
-                        for (int w = 0; w < 4; ++w) mw[w] = 0u;
+                        for (int i = 0; i < 2; ++i) {
+                            mw[i] = 0u;
 #pragma unroll
-                        for (int rr = 0; rr < 8; ++rr) {
-                            const int ky = st.y + rr;
-                            const int ady = abs(ky - q_y);
-                            uint32_t bits = 0u;
-                            if (q_valid && ky >= 0 && ky < prm.grid_h && ady < prm.n_half_width) {
-                                const int hw = half_width[ady];
-                                const int lo = max(max(q_x - hw, 0), st.x);
-                                const int hi = min(min(q_x + hw, prm.grid_w - 1), st.x + 15);
-                                if (lo <= hi) bits = ((1u << (hi - lo + 1)) - 1u) << (lo - st.x);
+                            for (int rr = 0; rr < 2; ++rr) {
+                                const int ky = org.y + 2 * (2 * i + hf) + rr;
+                                const int ady = abs(ky - q_y);
+                                uint32_t bits = 0u;
+                                if (q_valid && ky >= 0 && ky < prm.grid_h && ady < prm.n_half_width) {
+                                    const int hw = __ldg(prm.half_width + ady);
+                                    const int lo = max(max(q_x - hw, 0), org.x);
+                                    const int hi = min(min(q_x + hw, prm.grid_w - 1), org.x + 15);
+                                    if (lo <= hi) bits = ((1u << (hi - lo + 1)) - 1u) << (lo - org.x);
+                                }
+                                mw[i] |= bits << (16 * rr);
                             }
-                            mw[rr >> 1] |= bits << (16 * (rr & 1));
                         }
                     }
                 }
@@ -642,40 +672,56 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 }
                 ++n_s;
                 ptx::tc_fence_after();
-                uint32_t sv[4][32];
-#pragma unroll
-                for (int w = 0; w < 4; ++w) ptx::tmem_ld32(tmem_S + lane_off + 32 * w, sv[w]);
+                uint32_t sv[2][32];
+                ptx::tmem_ld32(tmem_S + lane_off, sv[0]);
+                ptx::tmem_ld32(tmem_S + lane_off + 64, sv[1]);
                 ptx::tmem_wait_ld();
                 // S_t is in registers: the next Q_t K^T may overwrite it
                 ptx::tc_fence_before();
                 warp_arrive(b_sfree, lane);
 
-                // row maximum over the allowed keys, four independent chains of three-input maxima
+                // maximum over this thread's allowed keys, four independent chains of three-input maxima
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 if (masked) {
 #pragma unroll
-                    for (int w = 0; w < 4; ++w)
+                    for (int i = 0; i < 2; ++i)
 #pragma unroll
                         for (int j = 0; j < 32; j += 2) {
-                            const float v0 = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
-                            const float v1 = ((mw[w] >> (j + 1)) & 1u) ? __uint_as_float(sv[w][j + 1]) : -INFINITY;
-                            sv[w][j] = __float_as_uint(v0);
-                            sv[w][j + 1] = __float_as_uint(v1);
+                            const float v0 = ((mw[i] >> j) & 1u) ? __uint_as_float(sv[i][j]) : -INFINITY;
+                            const float v1 = ((mw[i] >> (j + 1)) & 1u) ? __uint_as_float(sv[i][j + 1]) : -INFINITY;
+                            sv[i][j] = __float_as_uint(v0);
+                            sv[i][j + 1] = __float_as_uint(v1);
                             mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], v0, v1);
                         }
                 } else {
 #pragma unroll
-                    for (int w = 0; w < 4; ++w)
+                    for (int i = 0; i < 2; ++i)
 #pragma unroll
                         for (int j = 0; j < 32; j += 2)
-                            mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], __uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1]));
+                            mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], __uint_as_float(sv[i][j]), __uint_as_float(sv[i][j + 1]));
                 }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                // The row maximum only serves as the reference point of the exponentials: any value both
+                // threads of the row agree on will do, so it is exchanged rounded up to 16 bits.
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                {
+                    uint32_t bits = __float_as_uint(mx);
+                    bits = (mx > 0.f ? bits + 0xffffu : bits) & 0xffff0000u;
+                    uint16_t *xs = &ctrl->xchg[t][n_s & 1u][0][0];
+                    xs[hf * 128 + r] = (uint16_t)(bits >> 16);
+                    if (!pair_sync()) {
+                        alive = false;
+                        break;
+                    }
+                    const uint32_t other = (uint32_t)xs[(hf ^ 1) * 128 + r] << 16;
+                    mx = fmaxf(__uint_as_float(bits), __uint_as_float(other));
+                }
 
-                // Every P_t V issued so far must have retired before O_t is rescaled or the P buffer is
-                // written again (completion 2 i - 1 of the barrier: second half of the previous step).
+                if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
+
+                // The previous step's P_t V must have retired before O_t is rescaled or P is written again
+                // (the barrier completes once per step).
                 if (n_s > 1) {
-                    if (!__all_sync(0xffffffffu, wait_bar(b_pfree, 1u, abort_flag, prm.status, 17))) {
+                    if (!__all_sync(0xffffffffu, wait_bar(b_pfree, n_s & 1u, abort_flag, prm.status, 17))) {
                         alive = false;
                         break;
                     }
@@ -695,9 +741,9 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                             m_used = m_new;
                             l *= alpha;
                         }
-                        // S_t being ready means every earlier MMA, the last P_t V included, has retired
+                        // this thread's half of the output channels
 #pragma unroll 1
-                        for (int w = 0; w < D / 16; ++w) {
+                        for (int w = 0; w < kChan / 16; ++w) {
                             uint32_t o[16];
                             ptx::tmem_ld16(tmem_O + lane_off + 16 * w, o);
                             ptx::tmem_wait_ld();
@@ -705,43 +751,37 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                             for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
                             ptx::tmem_st16(tmem_O + lane_off + 16 * w, o);
                         }
+                        ptx::tmem_wait_st();
+                        ptx::tc_fence_before();
                     }
                 }
                 const float mc = (m_used == -INFINITY) ? 0.f : m_used * c;
 
-                // ---- P = exp2(S * c - m * c), row sum, bf16 pairs over the first 64 columns of S -----
+                // ---- P = exp2(S * c - m * c), row sum, bf16 pairs into the P half-tile ------------------
                 // (two-wide fp32 FMA and ADD; four independent partial sums)
                 const uint64_t c2 = ptx::pack2(c, c), nmc2 = ptx::pack2(-mc, -mc);
                 uint64_t lsum[2] = {0ull, 0ull};
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    // this half of the row (64 keys) as 32 bf16 pairs, kept in registers until the buffer is free
-                    uint32_t pk[32];
+                    // this thread's 32 keys of the half, 16 at a time (two 16-byte chunks of the row)
 #pragma unroll
-                    for (int w2 = 0; w2 < 2; ++w2) {
-                        const int w = 2 * h + w2;
+                    for (int grp = 0; grp < 2; ++grp) {
+                        uint32_t pk[8];
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
+                        for (int j = 16 * grp; j < 16 * grp + 16; j += 2) {
                             const uint64_t x2 =
-                                ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
+                                ptx::fma2(ptx::pack2(__uint_as_float(sv[h][j]), __uint_as_float(sv[h][j + 1])), c2, nmc2);
                             float x0, x1;
                             ptx::unpack2(x2, x0, x1);
                             const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
                             lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
-                            pk[16 * w2 + (j >> 1)] = ptx::pack_bf16(p0, p1);
+                            pk[(j >> 1) & 7] = ptx::pack_bf16(p0, p1);
                         }
-                    }
-                    if (h == 1) {
-                        // the first half's P_t V must have read the buffer (completion 2 i of the barrier)
-                        if (!__all_sync(0xffffffffu, wait_bar(b_pfree, 0u, abort_flag, prm.status, 18))) {
-                            alive = false;
-                            break;
-                        }
-                    }
 #pragma unroll
-                    for (int ch = 0; ch < 8; ++ch)
-                        *reinterpret_cast<uint4 *>(p_row + ((ch ^ (r & 7)) << 4)) =
-                            make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+                        for (int cc = 0; cc < 2; ++cc)
+                            *reinterpret_cast<uint4 *>(p_row + h * kHalfBytes + (((4 * hf + 2 * grp + cc) ^ (r & 7)) << 4)) =
+                                make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+                    }
                     // generic-proxy writes -> visible to the tensor core's (async proxy) reads
                     ptx::fence_proxy_async_smem();
                     warp_arrive(ptx::smem_u32(&ctrl->p_ready[t][h]), lane);
@@ -756,104 +796,76 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             }
             if (!alive) break;
 
-            // ---- hand the row statistics to the epilogue warps ------------------------------------
-            if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->stats_empty[t]), (n_items_seen & 1u) ^ 1u, abort_flag,
-                                                  prm.status, 11)))
+            // ---- epilogue: row sum of both threads, then O_t / l -> global memory ------------------------
+            // (hf = 1 hands its sum over, hf = 0 adds and hands the total back; the exchange slot not used
+            // by the last tile is free)
+            // The last P_t V has retired once o_full completes; by then every warp of the tile has also
+            // long read the row maxima of the last tile, so both exchange slots may be reused.
+            if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->o_full[t]), n_items_seen & 1u, abort_flag, prm.status, 14)))
                 break;
-            ctrl->stats[t][r] = make_float2(m_used * c, l);
-            warp_arrive(ptx::smem_u32(&ctrl->stats_full[t]), lane);
             ++n_items_seen;
-        }
-    } else {
-        // ================= epilogue warps: O_t / l -> global memory ========================================
-        ptx::setmaxnreg_dec<kRegsEpilogue>();
-        const int r = tid & 127;
-        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-        uint32_t n_seen[2] = {0, 0};
-        bool alive = true;
-        for (uint32_t k = 0; alive; ++k) {
-            const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
-            if (!__all_sync(0xffffffffu, wait_bar<500>(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 12)))
-                break;
-            const int g = ctrl->sched_item[slot];
-            const clear_pair_item_t item = ctrl->sched_rec[slot];
-            ItemRef ref;
-            ref.bh = ctrl->sched_bh[slot];
+            ptx::tc_fence_after();
+            {
+                float *mine = reinterpret_cast<float *>(&ctrl->xchg[t][hf][0][0]);
+                const float *other = reinterpret_cast<const float *>(&ctrl->xchg[t][hf ^ 1][0][0]);
+                mine[r] = l;
+                if (!pair_sync()) break;
+                const float lo = other[r];
+                l = hf == 0 ? l + lo : lo + l;  // the same sum, in the same order, in both threads
+                // nobody writes a row maximum of the next item into a slot before both have read this
+                if (!pair_sync()) break;
+            }
+            const int slot_p = t ? rec->partial_slot1 : rec->partial_slot0;
+            const int bh = ctrl->sched_bh[slot];
+            const int q_y = (t ? rec->qy1 : rec->qy0) + (r >> 4), q_x = rec->qx + (r & 15);
+            const long long token = is_text ? (long long)(rec->qx + t * 128 + r) : prm.n_text + (long long)q_y * prm.grid_w + q_x;
+            // the queue slot may be refilled now
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
-            if (g >= total_items) break;
-            for (int t = 0; t < item.n_sides; ++t) {
-                const uint32_t ph = n_seen[t] & 1u;
-                if (!__all_sync(0xffffffffu, wait_bar<500>(ptx::smem_u32(&ctrl->stats_full[t]), ph, abort_flag, prm.status, 13))) {
-                    alive = false;
-                    break;
-                }
-                const float2 ml = ctrl->stats[t][r];
-                warp_arrive(ptx::smem_u32(&ctrl->stats_empty[t]), lane);
-                if (!__all_sync(0xffffffffu, wait_bar<200>(ptx::smem_u32(&ctrl->o_full[t]), ph, abort_flag, prm.status, 14))) {
-                    alive = false;
-                    break;
-                }
-                ++n_seen[t];
-                ptx::tc_fence_after();
-                const uint32_t tmem_O = tmem + 256 + t * 128;
-                // which token is row r, and does it exist?
-                long long token;
-                bool q_valid;
-                if (item.kind == 1) {
-                    token = item.qx + t * 128 + r;
-                    q_valid = r < (t ? item.n_rows1 : item.n_rows0);
-                } else {
-                    const int q_y = (t ? item.qy1 : item.qy0) + (r >> 4), q_x = item.qx + (r & 15);
-                    q_valid = q_y < prm.grid_h && q_x < prm.grid_w;
-                    token = prm.n_text + (long long)q_y * prm.grid_w + q_x;
-                }
-                const int slot_p = t ? item.partial_slot1 : item.partial_slot0;
-                if (slot_p >= 0) {
-                    // split text-query tile: un-normalised fp32 row, its maximum (log2 units) and its sum
-                    const long long row = ((long long)ref.bh * prm.n_partial_slots + slot_p) * 128 + r;
-                    float *dst = prm.partial_o + row * D;
+            if (slot_p >= 0) {
+                // split text-query tile: un-normalised fp32 row, its maximum (log2 units) and its sum
+                const long long row = ((long long)bh * prm.n_partial_slots + slot_p) * 128 + r;
+                float *dst = prm.partial_o + row * D + kChan * hf;
 #pragma unroll
-                    for (int w = 0; w < D / 32; ++w) {
-                        uint32_t o[32];
-                        ptx::tmem_ld32(tmem_O + lane_off + 32 * w, o);
-                        ptx::tmem_wait_ld();
-                        if (w == D / 32 - 1) {
-                            ptx::tc_fence_before();
-                            warp_arrive(ptx::smem_u32(&ctrl->o_empty[t]), lane);
-                        }
-                        if (q_valid) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<uint4 *>(dst + 32 * w + j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
-                        }
+                for (int w = 0; w < kChan / 32; ++w) {
+                    uint32_t o[32];
+                    ptx::tmem_ld32(tmem_O + lane_off + 32 * w, o);
+                    ptx::tmem_wait_ld();
+                    if (w == kChan / 32 - 1) {
+                        ptx::tc_fence_before();
+                        warp_arrive(ptx::smem_u32(&ctrl->o_empty[t]), lane);
                     }
                     if (q_valid) {
-                        prm.partial_ml[row * 2] = ml.x;
-                        prm.partial_ml[row * 2 + 1] = ml.y;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<uint4 *>(dst + 32 * w + j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
                     }
-                } else {
-                    const float inv = ml.y > 0.f ? 1.f / ml.y : 0.f;
-                    __nv_bfloat16 *dst = prm.out + ((long long)ref.bh * prm.n_tokens + token) * D;
+                }
+                if (q_valid && hf == 0) {
+                    prm.partial_ml[row * 2] = m_used * c;
+                    prm.partial_ml[row * 2 + 1] = l;
+                }
+            } else {
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+                __nv_bfloat16 *dst = prm.out + ((long long)bh * prm.n_tokens + token) * D + kChan * hf;
 #pragma unroll
-                    for (int w = 0; w < D / 32; ++w) {
-                        uint32_t o[32];
-                        ptx::tmem_ld32(tmem_O + lane_off + 32 * w, o);
-                        ptx::tmem_wait_ld();
-                        if (w == D / 32 - 1) {
-                            ptx::tc_fence_before();
-                            warp_arrive(ptx::smem_u32(&ctrl->o_empty[t]), lane);
-                        }
-                        if (q_valid) {
+                for (int w = 0; w < kChan / 32; ++w) {
+                    uint32_t o[32];
+                    ptx::tmem_ld32(tmem_O + lane_off + 32 * w, o);
+                    ptx::tmem_wait_ld();
+                    if (w == kChan / 32 - 1) {
+                        ptx::tc_fence_before();
+                        warp_arrive(ptx::smem_u32(&ctrl->o_empty[t]), lane);
+                    }
+                    if (q_valid) {
 #pragma unroll
-                            for (int cc = 0; cc < 4; ++cc) {
-                                uint4 val;
-                                val.x = ptx::pack_bf16(__uint_as_float(o[8 * cc + 0]) * inv, __uint_as_float(o[8 * cc + 1]) * inv);
-                                val.y = ptx::pack_bf16(__uint_as_float(o[8 * cc + 2]) * inv, __uint_as_float(o[8 * cc + 3]) * inv);
-                                val.z = ptx::pack_bf16(__uint_as_float(o[8 * cc + 4]) * inv, __uint_as_float(o[8 * cc + 5]) * inv);
-                                val.w = ptx::pack_bf16(__uint_as_float(o[8 * cc + 6]) * inv, __uint_as_float(o[8 * cc + 7]) * inv);
-                                *reinterpret_cast<uint4 *>(dst + 32 * w + 8 * cc) = val;
-                            }
+                        for (int cc = 0; cc < 4; ++cc) {
+                            uint4 val;
+                            val.x = ptx::pack_bf16(__uint_as_float(o[8 * cc + 0]) * inv, __uint_as_float(o[8 * cc + 1]) * inv);
+                            val.y = ptx::pack_bf16(__uint_as_float(o[8 * cc + 2]) * inv, __uint_as_float(o[8 * cc + 3]) * inv);
+                            val.z = ptx::pack_bf16(__uint_as_float(o[8 * cc + 4]) * inv, __uint_as_float(o[8 * cc + 5]) * inv);
+                            val.w = ptx::pack_bf16(__uint_as_float(o[8 * cc + 6]) * inv, __uint_as_float(o[8 * cc + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(dst + 32 * w + 8 * cc) = val;
                         }
                     }
                 }
@@ -950,7 +962,7 @@ std::mutex g_dev_mutex;
 template <int D>
 int launch_variant(const clear_plan &p, const CUtensorMap *tm, const WsParams &prm, cudaStream_t stream)
 {
-    constexpr size_t kSmem = (size_t)(2 + kRing) * (D / 64) * 16384 + 2 * 16384 + sizeof(Ctrl);
+    constexpr size_t kSmem = (size_t)(2 + kRing) * (D / 64) * 16384 + 4 * 16384 + sizeof(Ctrl);
     static_assert(kSmem <= 232448, "shared memory of one block");
     int n_sm = 0;
     {

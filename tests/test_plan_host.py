@@ -250,10 +250,23 @@ def test_pair_schedule_covers_each_allowed_pair_exactly_once(gh, gw, T, r):
     for it in items:
         assert it.step_count >= 1 and it.n_sides in (1, 2)
         sts = steps[it.step_begin: it.step_begin + it.step_count]
-        # ring bookkeeping: K and V of each distinct key tile of a step take one stage each
+        # ring bookkeeping: K and V of each distinct key tile of a step take one stage each, in the order
+        # K(0), then K(s + 1), V(s) for every step s
+        def tiles_of(st):
+            return int(bool(st.flags & clear.STEP_USE0)) + int(bool(st.flags & clear.STEP_USE1) and
+                                                               not st.flags & clear.STEP_SHARED)
+        order = [("K", 0)]
+        for i in range(len(sts)):
+            if i + 1 < len(sts):
+                order.append(("K", i + 1))
+            order.append(("V", i))
+        pos, where = 0, {}
+        for kind, i in order:
+            where[(kind, i)] = pos
+            pos += tiles_of(sts[i])
         loads = 0
-        for st in sts:
-            assert st.load_base == loads
+        for i, st in enumerate(sts):
+            assert st.load_base & 0xffff == where[("K", i)] and st.load_base >> 16 == where[("V", i)]
             use0, use1 = bool(st.flags & clear.STEP_USE0), bool(st.flags & clear.STEP_USE1)
             shared = bool(st.flags & clear.STEP_SHARED)
             assert use0 or use1
