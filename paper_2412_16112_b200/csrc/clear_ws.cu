@@ -5,18 +5,17 @@
 // text tokens -- and a list of steps; in each step every query tile of the pair meets one 128-key
 // tile (Eq. 1 restricted by Eq. 3).  Key tiles both query tiles need are staged once.
 //
-// Roles (640 threads):
+// Roles (384 threads):
 //   warp 0        : takes items from the queue and issues every TMA load (Q tiles, K/V ring);
 //   warps 1, 2    : one thread each issues the tcgen05.mma of query tile t = 0, 1: S_t = Q_t K^T,
 //                   O_t += P_t V; the softmax of one query tile runs under the MMAs of the other;
-//   warps 4-11    : softmax and epilogue of query tile 0, two threads per query row (= tensor-memory
-//                   lane), each with half of the keys of every tile: mask, maximum, P = exp2(.) as bf16
-//                   into shared memory, row sum; at the end of an item O / l -> bf16 -> global memory
-//                   (or fp32 partial results of split text rows);
-//   warps 12-19   : the same for query tile 1.
+//   warps 4-7     : softmax and epilogue of query tile 0 (thread r owns query row r = tensor-memory
+//                   lane r): mask, running maximum, P = exp2(.) as bf16 into shared memory, row sum; at the
+//                   end of an item O / l -> bf16 -> global memory (or fp32 partial results of split text
+//                   rows);
+//   warps 8-11    : the same for query tile 1.
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each.  P goes through shared memory, so
-// that S_t of the next step can be computed while the softmax of this one runs; it is handed to the
-// tensor core 64 keys at a time.
+// that S_t of the next step can be computed while the softmax of this one runs.
 // Shared memory: Q0, Q1, a ring of three key/value stages (K and V tiles take one stage each) and P
 // of each query tile.
 // Every wait is bounded: on expiry the block raises the plan's status word and leaves.
@@ -32,7 +31,7 @@
 namespace clear {
 namespace {
 
-constexpr int kWsThreads = 640;   // 4 control warps + 2 x 8 softmax warps
+constexpr int kWsThreads = 384;   // 4 control warps + 2 x 4 softmax warps
 constexpr int kRing = 3;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -40,11 +39,11 @@ constexpr uint32_t kWaitHintNs = 20000;            // one sleep inside try_wait
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the row max grows by more
 constexpr int kSchedDepth = 2;
-// arrivals that free a queue slot: the two MMA threads and one lane of each of the 16 softmax warps
-constexpr uint32_t kSchedReaders = 18;
-// registers per thread of each role: 128 x 64 + 512 x 104 = 61440 = what the block is launched with
-// (640 threads x 96); raising a warp's budget only draws on registers other warps of the block gave back
-constexpr uint32_t kRegsControl = 64, kRegsSoftmax = 104;
+// arrivals that free a queue slot: the two MMA threads and one lane of each of the 8 softmax warps
+constexpr uint32_t kSchedReaders = 10;
+// registers per thread of each role: 128 x 64 + 256 x 216 = 63488, within what the block is launched with
+// (384 threads x 168); raising a warp's budget only draws on registers other warps of the block gave back
+constexpr uint32_t kRegsControl = 64, kRegsSoftmax = 216;
 
 struct WsParams {
     const clear_pair_item_t *items;
@@ -66,8 +65,7 @@ struct WsParams {
 struct Ctrl {
     uint64_t q_full[2], q_empty[2];
     uint64_t kv_full[kRing], kv_empty[kRing];
-    uint64_t s_full[2], s_free[2], p_ready[2][2], p_free[2], o_full[2], o_empty[2];
-    uint64_t pair[2][4];  // the two warps that share 32 query rows of a tile
+    uint64_t s_full[2], s_free[2], p_ready[2], p_free[2], o_full[2], o_empty[2];
     uint64_t sched_full[kSchedDepth], sched_empty[kSchedDepth];
     uint64_t drain[2];
     int32_t sched_item[kSchedDepth];            // queue position, >= total: no more work
@@ -76,9 +74,6 @@ struct Ctrl {
     uint32_t tmem_base;
     int abort_flag;
     int skip;
-    // [query tile][slot][thread of the row][row]: the row maxima (16 bits each) the two threads of a row
-    // show each other, two slots used in turn; at the end of an item each slot holds 128 fp32 row sums
-    alignas(16) uint16_t xchg[2][2][2][128];
 };
 
 // Bounded wait on an mbarrier phase.  Returns false once the block has given up.  The polling loop is
@@ -244,13 +239,11 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_empty[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->s_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->s_free[i]), 8);  // one arrival per softmax warp of the tile
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][0]), 8);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i][1]), 8);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->s_free[i]), 4);  // one arrival per softmax warp of the tile
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i]), 4);
             ptx::mbar_init(ptx::smem_u32(&ctrl->p_free[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->o_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 8);
-            for (int j = 0; j < 4; ++j) ptx::mbar_init(ptx::smem_u32(&ctrl->pair[i][j]), 2);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 4);
         }
         for (int i = 0; i < kRing; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->kv_full[i]), 1);
@@ -483,14 +476,14 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         }
                     }
 
-                    // O_t += P_t V, 64 keys at a time as the softmax warps deliver P's halves
+                    // O_t += P_t V, the two 64-key halves of P one after the other
                     if (!qk_done) kv_walk(pos_v, kNone);
                     uint32_t stage_v = 0;
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        ok = wait_bar(ptx::smem_u32(&ctrl->p_ready[t][h]), n_pv & 1u, abort_flag, prm.status, 7);
-                        if (!ok) break;
                         if (h == 0) {
+                            ok = wait_bar(ptx::smem_u32(&ctrl->p_ready[t]), n_pv & 1u, abort_flag, prm.status, 7);
+                            if (!ok) break;
                             stage_v = kv_wait(pos_v, kNone);
                             if (!ok) break;
                             if (first_pv) {
@@ -537,130 +530,111 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         }
         __syncwarp();
     } else {
-        // ================= softmax warps ===================================================================
-        // Eight warps per query tile, two threads per query row (tensor-memory lane): the thread with
-        // hf = 0 takes keys [0, 32) and [64, 96) of every 128-key tile, its partner (hf = 1, four warps
-        // further on) keys [32, 64) and [96, 128).  Four such warps per scheduler hide each other's
-        // instruction latencies.  The two threads of a row agree on the row maximum through shared
-        // memory once per tile and add up their row sums once per item; each normalises and stores half
-        // of the output channels.
+        // ================= softmax warps: thread r owns query row r (tensor-memory lane r) of its tile =====
+        // Per step: S_t into registers (the next Q_t K^T may then overwrite it), Eq. 3 mask, row maximum,
+        // P = exp2(.) as bf16 into shared memory with the row sum; at the end of an item O_t / l -> bf16 ->
+        // global memory (or fp32 partial results of split text rows).
         ptx::setmaxnreg_inc<kRegsSoftmax>();
-        const int ws = warp - 4;
-        const int t = ws >> 3;          // query tile of the pair
-        const int hf = (ws >> 2) & 1;
-        const int q4 = ws & 3;          // tensor-memory lane quadrant (= warp % 4)
+        const int t = (warp - 4) >> 2;  // query tile of the pair
+        const int q4 = warp & 3;        // tensor-memory lane quadrant
         const int r = q4 * 32 + lane;   // query row of the tile
-        constexpr int kChan = D / 2;    // output channels per thread
         const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
-        const uint32_t tmem_S = tmem + t * 128 + 32 * hf, tmem_O = tmem + 256 + t * 128 + kChan * hf;
+        const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
         const float c = prm.scale_log2;
         const uint32_t b_s = ptx::smem_u32(&ctrl->s_full[t]), b_sfree = ptx::smem_u32(&ctrl->s_free[t]);
-        const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]);
-        const uint32_t b_pair = ptx::smem_u32(&ctrl->pair[t][q4]);
-        // this thread's 64 bytes of its row of the P half-tile: K-major, 128-byte rows, 16-byte chunks
+        const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]), b_pready = ptx::smem_u32(&ctrl->p_ready[t]);
+        // this row of the two P half-tiles (64 keys each): K-major, 128-byte rows, 16-byte chunks
         // XOR-swizzled by the row number
         uint8_t *p_row = smem_raw + (sP - smem_base) + t * 2 * kHalfBytes + r * 128;
-        uint32_t n_s = 0, n_pair = 0, n_items_seen = 0;
+        uint32_t n_s = 0, n_items_seen = 0;
         bool alive = true;
-        // the two warps of a row meet: one arrival each, then both see what the other wrote before
-        auto pair_sync = [&]() -> bool {
-            warp_arrive(b_pair, lane);
-            const bool ok = __all_sync(0xffffffffu, wait_bar(b_pair, n_pair & 1u, abort_flag, prm.status, 19));
-            ++n_pair;
-            return ok;
-        };
         for (uint32_t k = 0; alive; ++k) {
             const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
             if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 9)))
                 break;
             const int g = ctrl->sched_item[slot];
-            // The item's record stays in its queue slot until this warp is done with the item (the slot
-            // is given back at the end), so that only what every step needs lives in registers.
-            const volatile clear_pair_item_t *rec = &ctrl->sched_rec[slot];
-            if (g >= total_items || t >= rec->n_sides) {
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
-                if (g >= total_items) break;
-                continue;
-            }
-            const clear_pair_step_t *steps = prm.steps + rec->step_begin;
-            const int step_count = rec->step_count;
-            const bool is_text = rec->kind == 1;
-            // does this row's query exist?  (image tiles: its grid position lies on the grid)
-            bool q_valid;
-            {
-                const int q_y = (t ? rec->qy1 : rec->qy0) + (r >> 4), q_x = rec->qx + (r & 15);
-                q_valid = is_text ? r < (t ? rec->n_rows1 : rec->n_rows0) : (q_y < prm.grid_h && q_x < prm.grid_w);
-            }
+            const clear_pair_item_t item = ctrl->sched_rec[slot];
+            const int bh = ctrl->sched_bh[slot];
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
+            if (g >= total_items) break;
+            if (t >= item.n_sides) continue;
+            const clear_pair_step_t *steps = prm.steps + item.step_begin;
+            const int step_count = item.step_count;
+            const bool is_text = item.kind == 1;
+            // grid position of this row's query (image tiles), and whether the row exists
+            const int q_y = (t ? item.qy1 : item.qy0) + (r >> 4), q_x = item.qx + (r & 15);
+            const bool q_valid = is_text ? r < (t ? item.n_rows1 : item.n_rows0) : (q_y < prm.grid_h && q_x < prm.grid_w);
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
 
             // The next step's record is fetched at the top of a step and this row's precomputed mask words
             // for it in the middle, so that neither latency is on the critical path.
             const int kMaskedBit = t ? CLEAR_STEP_MASKED1 : CLEAR_STEP_MASKED0;
-            auto load_mask_row = [&](const SideStep &q) -> uint2 {
-                if (step_uses(q.flags, t) && (q.flags & kMaskedBit) && !(q.flags & CLEAR_STEP_LINEAR) && q.n_valid >= 0) {
-                    const uint32_t *e = prm.mask_table + ((size_t)q.n_valid * 128 + r) * 4 + hf;
-                    return make_uint2(__ldg(e), __ldg(e + 2));
-                }
-                return make_uint2(0u, 0u);
+            auto load_mask_row = [&](const SideStep &q) -> uint4 {
+                if (step_uses(q.flags, t) && (q.flags & kMaskedBit) && !(q.flags & CLEAR_STEP_LINEAR) && q.n_valid >= 0)
+                    return __ldg(reinterpret_cast<const uint4 *>(prm.mask_table) + ((size_t)q.n_valid * 128 + r));
+                return make_uint4(0u, 0u, 0u, 0u);
             };
             SideStep st_next = load_side_step(steps, t);
-            uint2 mrow_next = load_mask_row(st_next);
+            uint4 mrow_next = load_mask_row(st_next);
             for (int s = 0; s < step_count; ++s) {
                 const SideStep st = st_next;
-                const uint2 mrow = mrow_next;
+                const uint4 mrow = mrow_next;
                 if (s + 1 < step_count) st_next = load_side_step(steps + s + 1, t);
                 if (!step_uses(st.flags, t)) {
                     if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
                     continue;
                 }
                 const bool masked = (st.flags & kMaskedBit) != 0;
-                // ---- mask bits of this thread's keys: mw[i] bit j = key 64 i + 32 hf + j allowed -------
-                uint32_t mw[2] = {0xffffffffu, 0xffffffffu};
+                // ---- mask bits of this row for the tile (bit j of word w = key 32 w + j allowed) --------
+                uint32_t mw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
                 if (masked) {
                     if (st.flags & CLEAR_STEP_LINEAR) {
 #pragma unroll
-                        for (int i = 0; i < 2; ++i) {
-                            const int nv = min(max(st.n_valid - 32 * (2 * i + hf), 0), 32);
-                            mw[i] = nv == 32 ? 0xffffffffu : ((1u << nv) - 1u);
+                        for (int w = 0; w < 4; ++w) {
+                            const int nv = min(max(st.n_valid - 32 * w, 0), 32);
+                            mw[w] = nv == 32 ? 0xffffffffu : ((1u << nv) - 1u);
                         }
                     } else if (st.n_valid >= 0) {
                         // Eq. 3 from the table; keys of the patch that lie off the grid do not exist
                         mw[0] = mrow.x;
                         mw[1] = mrow.y;
+                        mw[2] = mrow.z;
+                        mw[3] = mrow.w;
                         if (st.flags & (t ? CLEAR_STEP_CLIP1 : CLEAR_STEP_CLIP0)) {
                             const int2 org = load_side_origin(steps + s, t);
                             const int lo = max(0, -org.x), hi = min(15, prm.grid_w - 1 - org.x);
                             const uint32_t cols = lo <= hi ? (((1u << (hi - lo + 1)) - 1u) << lo) : 0u;
 #pragma unroll
-                            for (int i = 0; i < 2; ++i) {
-                                const int ky0 = org.y + 2 * (2 * i + hf), ky1 = ky0 + 1;
+                            for (int w = 0; w < 4; ++w) {
+                                const int ky0 = org.y + 2 * w, ky1 = ky0 + 1;
                                 const uint32_t ok0 = (ky0 >= 0 && ky0 < prm.grid_h) ? cols : 0u;
                                 const uint32_t ok1 = (ky1 >= 0 && ky1 < prm.grid_h) ? cols : 0u;
-                                mw[i] &= ok0 | (ok1 << 16);
+                                mw[w] &= ok0 | (ok1 << 16);
                             }
                         }
                     } else {
                         // no table entry (very large radius): Eq. 3 row by row from the half widths
                         const int2 org = load_side_origin(steps + s, t);
-                        const int q_y = (t ? rec->qy1 : rec->qy0) + (r >> 4), q_x = rec->qx + (r & 15);
 #pragma unroll
-                        for (int i = 0; i < 2; ++i) {
-                            mw[i] = 0u;
-#pragma unroll
-                            for (int rr = 0; rr < 2; ++rr) {
-                                const int ky = org.y + 2 * (2 * i + hf) + rr;
-                                const int ady = abs(ky - q_y);
-                                uint32_t bits = 0u;
-                                if (q_valid && ky >= 0 && ky < prm.grid_h && ady < prm.n_half_width) {
-                                    const int hw = __ldg(prm.half_width + ady);
-                                    const int lo = max(max(q_x - hw, 0), org.x);
-                                    const int hi = min(min(q_x + hw, prm.grid_w - 1), org.x + 15);
-                                    if (lo <= hi) bits = ((1u << (hi - lo + 1)) - 1u) << (lo - org.x);
-                                }
-                                mw[i] |= bits << (16 * rr);
+                        for (int w = 0; w < 4; ++w) mw[w] = 0u;
+#pragma unroll 1
+                        for (int rr = 0; rr < 8; ++rr) {
+                            const int ky = org.y + rr;
+                            const int ady = abs(ky - q_y);
+                            uint32_t bits = 0u;
+                            if (q_valid && ky >= 0 && ky < prm.grid_h && ady < prm.n_half_width) {
+                                const int hw = __ldg(prm.half_width + ady);
+                                const int lo = max(max(q_x - hw, 0), org.x);
+                                const int hi = min(min(q_x + hw, prm.grid_w - 1), org.x + 15);
+                                if (lo <= hi) bits = ((1u << (hi - lo + 1)) - 1u) << (lo - org.x);
                             }
+                            bits <<= 16 * (rr & 1);
+                            if ((rr >> 1) == 0) mw[0] |= bits;
+                            if ((rr >> 1) == 1) mw[1] |= bits;
+                            if ((rr >> 1) == 2) mw[2] |= bits;
+                            if ((rr >> 1) == 3) mw[3] |= bits;
                         }
                     }
                 }
@@ -672,51 +646,36 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 }
                 ++n_s;
                 ptx::tc_fence_after();
-                uint32_t sv[2][32];
-                ptx::tmem_ld32(tmem_S + lane_off, sv[0]);
-                ptx::tmem_ld32(tmem_S + lane_off + 64, sv[1]);
+                uint32_t sv[4][32];
+#pragma unroll
+                for (int w = 0; w < 4; ++w) ptx::tmem_ld32(tmem_S + lane_off + 32 * w, sv[w]);
                 ptx::tmem_wait_ld();
                 // S_t is in registers: the next Q_t K^T may overwrite it
                 ptx::tc_fence_before();
                 warp_arrive(b_sfree, lane);
+                if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
 
-                // maximum over this thread's allowed keys, four independent chains of three-input maxima
+                // row maximum over the allowed keys, four independent chains of three-input maxima
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 if (masked) {
 #pragma unroll
-                    for (int i = 0; i < 2; ++i)
+                    for (int w = 0; w < 4; ++w)
 #pragma unroll
                         for (int j = 0; j < 32; j += 2) {
-                            const float v0 = ((mw[i] >> j) & 1u) ? __uint_as_float(sv[i][j]) : -INFINITY;
-                            const float v1 = ((mw[i] >> (j + 1)) & 1u) ? __uint_as_float(sv[i][j + 1]) : -INFINITY;
-                            sv[i][j] = __float_as_uint(v0);
-                            sv[i][j + 1] = __float_as_uint(v1);
+                            const float v0 = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
+                            const float v1 = ((mw[w] >> (j + 1)) & 1u) ? __uint_as_float(sv[w][j + 1]) : -INFINITY;
+                            sv[w][j] = __float_as_uint(v0);
+                            sv[w][j + 1] = __float_as_uint(v1);
                             mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], v0, v1);
                         }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 2; ++i)
+                    for (int w = 0; w < 4; ++w)
 #pragma unroll
                         for (int j = 0; j < 32; j += 2)
-                            mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], __uint_as_float(sv[i][j]), __uint_as_float(sv[i][j + 1]));
+                            mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], __uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1]));
                 }
-                // The row maximum only serves as the reference point of the exponentials: any value both
-                // threads of the row agree on will do, so it is exchanged rounded up to 16 bits.
-                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                {
-                    uint32_t bits = __float_as_uint(mx);
-                    bits = (mx > 0.f ? bits + 0xffffu : bits) & 0xffff0000u;
-                    uint16_t *xs = &ctrl->xchg[t][n_s & 1u][0][0];
-                    xs[hf * 128 + r] = (uint16_t)(bits >> 16);
-                    if (!pair_sync()) {
-                        alive = false;
-                        break;
-                    }
-                    const uint32_t other = (uint32_t)xs[(hf ^ 1) * 128 + r] << 16;
-                    mx = fmaxf(__uint_as_float(bits), __uint_as_float(other));
-                }
-
-                if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
 
                 // The previous step's P_t V must have retired before O_t is rescaled or P is written again
                 // (the barrier completes once per step).
@@ -741,9 +700,8 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                             m_used = m_new;
                             l *= alpha;
                         }
-                        // this thread's half of the output channels
 #pragma unroll 1
-                        for (int w = 0; w < kChan / 16; ++w) {
+                        for (int w = 0; w < D / 16; ++w) {
                             uint32_t o[16];
                             ptx::tmem_ld16(tmem_O + lane_off + 16 * w, o);
                             ptx::tmem_wait_ld();
@@ -757,20 +715,19 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 }
                 const float mc = (m_used == -INFINITY) ? 0.f : m_used * c;
 
-                // ---- P = exp2(S * c - m * c), row sum, bf16 pairs into the P half-tile ------------------
+                // ---- P = exp2(S * c - m * c), row sum, bf16 pairs into the P half-tiles -----------------
                 // (two-wide fp32 FMA and ADD; four independent partial sums)
                 const uint64_t c2 = ptx::pack2(c, c), nmc2 = ptx::pack2(-mc, -mc);
                 uint64_t lsum[2] = {0ull, 0ull};
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    // this thread's 32 keys of the half, 16 at a time (two 16-byte chunks of the row)
+                for (int w = 0; w < 4; ++w) {
 #pragma unroll
                     for (int grp = 0; grp < 2; ++grp) {
-                        uint32_t pk[8];
+                        uint32_t pk[8];  // 16 keys = two 16-byte chunks of the row
 #pragma unroll
                         for (int j = 16 * grp; j < 16 * grp + 16; j += 2) {
                             const uint64_t x2 =
-                                ptx::fma2(ptx::pack2(__uint_as_float(sv[h][j]), __uint_as_float(sv[h][j + 1])), c2, nmc2);
+                                ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
                             float x0, x1;
                             ptx::unpack2(x2, x0, x1);
                             const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
@@ -778,15 +735,16 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                             pk[(j >> 1) & 7] = ptx::pack_bf16(p0, p1);
                         }
 #pragma unroll
-                        for (int cc = 0; cc < 2; ++cc)
-                            *reinterpret_cast<uint4 *>(p_row + h * kHalfBytes + (((4 * hf + 2 * grp + cc) ^ (r & 7)) << 4)) =
+                        for (int cc = 0; cc < 2; ++cc) {
+                            const int ch = 4 * (w & 1) + 2 * grp + cc;  // chunk of the 128-byte row of half w / 2
+                            *reinterpret_cast<uint4 *>(p_row + (w >> 1) * kHalfBytes + ((ch ^ (r & 7)) << 4)) =
                                 make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+                        }
                     }
-                    // generic-proxy writes -> visible to the tensor core's (async proxy) reads
-                    ptx::fence_proxy_async_smem();
-                    warp_arrive(ptx::smem_u32(&ctrl->p_ready[t][h]), lane);
                 }
-                if (!alive) break;
+                // generic-proxy writes -> visible to the tensor core's (async proxy) reads
+                ptx::fence_proxy_async_smem();
+                warp_arrive(b_pready, lane);
                 {
                     float a0, a1, a2, a3;
                     ptx::unpack2(lsum[0], a0, a1);
@@ -796,42 +754,22 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             }
             if (!alive) break;
 
-            // ---- epilogue: row sum of both threads, then O_t / l -> global memory ------------------------
-            // (hf = 1 hands its sum over, hf = 0 adds and hands the total back; the exchange slot not used
-            // by the last tile is free)
-            // The last P_t V has retired once o_full completes; by then every warp of the tile has also
-            // long read the row maxima of the last tile, so both exchange slots may be reused.
+            // ---- epilogue: the last P_t V has retired once o_full completes; O_t / l -> global memory -----
             if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->o_full[t]), n_items_seen & 1u, abort_flag, prm.status, 14)))
                 break;
             ++n_items_seen;
             ptx::tc_fence_after();
-            {
-                float *mine = reinterpret_cast<float *>(&ctrl->xchg[t][hf][0][0]);
-                const float *other = reinterpret_cast<const float *>(&ctrl->xchg[t][hf ^ 1][0][0]);
-                mine[r] = l;
-                if (!pair_sync()) break;
-                const float lo = other[r];
-                l = hf == 0 ? l + lo : lo + l;  // the same sum, in the same order, in both threads
-                // nobody writes a row maximum of the next item into a slot before both have read this
-                if (!pair_sync()) break;
-            }
-            const int slot_p = t ? rec->partial_slot1 : rec->partial_slot0;
-            const int bh = ctrl->sched_bh[slot];
-            const int q_y = (t ? rec->qy1 : rec->qy0) + (r >> 4), q_x = rec->qx + (r & 15);
-            const long long token = is_text ? (long long)(rec->qx + t * 128 + r) : prm.n_text + (long long)q_y * prm.grid_w + q_x;
-            // the queue slot may be refilled now
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
+            const int slot_p = t ? item.partial_slot1 : item.partial_slot0;
             if (slot_p >= 0) {
                 // split text-query tile: un-normalised fp32 row, its maximum (log2 units) and its sum
                 const long long row = ((long long)bh * prm.n_partial_slots + slot_p) * 128 + r;
-                float *dst = prm.partial_o + row * D + kChan * hf;
+                float *dst = prm.partial_o + row * D;
 #pragma unroll
-                for (int w = 0; w < kChan / 32; ++w) {
+                for (int w = 0; w < D / 32; ++w) {
                     uint32_t o[32];
                     ptx::tmem_ld32(tmem_O + lane_off + 32 * w, o);
                     ptx::tmem_wait_ld();
-                    if (w == kChan / 32 - 1) {
+                    if (w == D / 32 - 1) {
                         ptx::tc_fence_before();
                         warp_arrive(ptx::smem_u32(&ctrl->o_empty[t]), lane);
                     }
@@ -841,19 +779,20 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                             *reinterpret_cast<uint4 *>(dst + 32 * w + j) = make_uint4(o[j], o[j + 1], o[j + 2], o[j + 3]);
                     }
                 }
-                if (q_valid && hf == 0) {
+                if (q_valid) {
                     prm.partial_ml[row * 2] = m_used * c;
                     prm.partial_ml[row * 2 + 1] = l;
                 }
             } else {
                 const float inv = l > 0.f ? 1.f / l : 0.f;
-                __nv_bfloat16 *dst = prm.out + ((long long)bh * prm.n_tokens + token) * D + kChan * hf;
+                const long long token = is_text ? (long long)(item.qx + t * 128 + r) : prm.n_text + (long long)q_y * prm.grid_w + q_x;
+                __nv_bfloat16 *dst = prm.out + ((long long)bh * prm.n_tokens + token) * D;
 #pragma unroll
-                for (int w = 0; w < kChan / 32; ++w) {
+                for (int w = 0; w < D / 32; ++w) {
                     uint32_t o[32];
                     ptx::tmem_ld32(tmem_O + lane_off + 32 * w, o);
                     ptx::tmem_wait_ld();
-                    if (w == kChan / 32 - 1) {
+                    if (w == D / 32 - 1) {
                         ptx::tc_fence_before();
                         warp_arrive(ptx::smem_u32(&ctrl->o_empty[t]), lane);
                     }
