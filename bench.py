@@ -111,7 +111,7 @@ def allowed_counts(w):
     return _COUNTS_CACHE[key]
 
 
-def time_oracle_sample(w, q, k, v, target_s=12.0):
+def time_oracle_sample(w, q, k, v, target_s=15.0):
     """Oracle throughput on a bounded sample of query rows of head 0, in the metric's unit:
     4 * (allowed pairs of the sampled rows) * head_dim / seconds."""
     from oracle import clear_oracle as oracle
@@ -257,12 +257,16 @@ def run_ours(args, w):
     # ---- roofline of the dominant kernel ------------------------------------------------------------
     per_gpu_tflops = flops / (ms_per_step * 1e-3) / 1e12
     peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+    # DRAM bytes of one launch from the committed ncu capture (profiles/): "workload bytes" per line
     traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.txt")
+    if os.path.exists(tpath) and info.kernel == clear.KERNEL_TCGEN05_WS:
         try:
             with open(tpath) as f:
-                traffic = json.load(f).get(w.name)
+                for line in f:
+                    parts = line.split()
+                    if len(parts) == 2 and parts[0] == w.name:
+                        traffic = float(parts[1])
         except Exception:
             traffic = None
     if info.kernel != clear.KERNEL_SIMT:
