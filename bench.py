@@ -123,10 +123,16 @@ def time_oracle_sample(w, q, k, v, target_s=15.0):
     scale_up = max(1.0, target_s / max(t_pilot, 1e-3))
     n_text_rows = max(2, int(2 * scale_up))
     n_img_rows = max(64, int(64 * scale_up))
-    rows = sample_rows_for_cpu(w, n_text_rows, n_img_rows, seed=1)
-    t0 = time.perf_counter()
-    oracle.attn_rows(q, k, v, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale, rows)
-    dt = time.perf_counter() - t0
+    # the pilot includes one-off costs, so it underestimates the rate: grow the sample until it runs long enough
+    for attempt in range(3):
+        rows = sample_rows_for_cpu(w, n_text_rows, n_img_rows, seed=1)
+        t0 = time.perf_counter()
+        oracle.attn_rows(q, k, v, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale, rows)
+        dt = time.perf_counter() - t0
+        if dt >= 0.6 * target_s:
+            break
+        grow = min(8.0, target_s / max(dt, 1e-3))
+        n_text_rows, n_img_rows = int(n_text_rows * grow), int(n_img_rows * grow)
     pairs = int(counts[rows[:, 2]].sum())
     tflops = 4.0 * pairs * w.head_dim / dt / 1e12
     return {"value": tflops, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
