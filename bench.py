@@ -165,6 +165,20 @@ def run_reference(args, w):
     return 0
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time: the replicas of a multi-GPU run are as fast as their slowest member."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(world: int, flops_per_replica: float, ms_per_step: float) -> float:
+    """Whole-job TFLOP/s of `world` independent replicas that all take `ms_per_step` (the slowest rank's)."""
+    return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
+
+
 def workload_config(w):
     return {"workload": w.name, "B": w.B, "H": w.H, "head_dim": w.head_dim, "grid_h": w.grid_h, "grid_w": w.grid_w,
             "n_text": w.n_text, "radius": w.radius, "l2": "inputs larger than L2 (no flush)" if
@@ -223,13 +237,9 @@ def run_ours(args, w):
         t_wall = time.perf_counter() - t_wall0
     plan.check()
     ms = [a.elapsed_time(b) for a, b in ev]
-    total_ms = float(sum(ms))
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(float(sum(ms)), dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    value = replica_throughput(world, flops, ms_per_step)
     clock_info = clocks.summary()
 
     # ---- end to end: host tensors in pinned memory, copies inside the timed region ----------------
@@ -246,13 +256,9 @@ def run_ours(args, w):
             plan.forward_host(qh, kh, vh, oh, w.scale)
         e1.record(stream)
         barrier()
-        e2e_ms = e0.elapsed_time(e1) / n_e2e
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1) / n_e2e, dist, dev)
         nbytes = q.numel() * q.element_size()
-        e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+        e2e = {"value": replica_throughput(world, flops, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes, "steps": n_e2e}
 
     if rank != 0:
