@@ -377,17 +377,17 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             // after both arrivals, so neither thread ever waits on a barrier phase that is more than one
             // ahead of the barrier (mbarrier waits tell phases apart by one parity bit only).
             uint32_t next_pos = 0;  // first position whose fill this thread has not seen yet
-            // see the fills of [next_pos, pos) and free them at once, except `keep` (a V tile still to be read)
-            auto kv_walk = [&](uint32_t pos, uint32_t keep) {
+            // see the fills of [next_pos, pos), stages this thread does not read, and free them at once
+            auto kv_walk = [&](uint32_t pos) {
                 for (; next_pos < pos && ok; ++next_pos) {
                     const uint32_t st = next_pos % kRing, fl = next_pos / kRing;
                     ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[st]), fl & 1u, abort_flag, prm.status, 15);
-                    if (ok && next_pos != keep) ptx::mbar_arrive(ptx::smem_u32(&ctrl->kv_empty[st]));
+                    if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->kv_empty[st]));
                 }
             };
             // wait for the fill of `pos`, a stage this thread reads
-            auto kv_wait = [&](uint32_t pos, uint32_t keep) -> uint32_t {
-                kv_walk(pos, keep);
+            auto kv_wait = [&](uint32_t pos) -> uint32_t {
+                kv_walk(pos);
                 const uint32_t stage = pos % kRing, fill = pos / kRing;
                 if (ok && next_pos == pos) {
                     ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[stage]), fill & 1u, abort_flag, prm.status, 4);
@@ -396,7 +396,6 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 return stage;
             };
             auto kv_release = [&](uint32_t stage) { ptx::tc_commit(ptx::smem_u32(&ctrl->kv_empty[stage])); };
-            constexpr uint32_t kNone = 0xffffffffu;
             for (uint32_t k = 0; ok; ++k) {
                 const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
                 if (!wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 5)) break;
@@ -406,7 +405,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 if (g >= total_items) break;
                 if (t >= item.n_sides) {
                     ring_base += (uint32_t)item.n_loads;
-                    kv_walk(ring_base, kNone);
+                    kv_walk(ring_base);
                     continue;
                 }
                 const clear_pair_step_t *steps = prm.steps + item.step_begin;
@@ -416,13 +415,12 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
 
                 // S_t = Q_t K^T for the key tile of `st`; both operands K-major: 16 contraction channels
                 // are 32 bytes along a 128-byte row, the next 64 channels are the tile's second half.
-                // `keep`: position of a V tile this thread still has to read (or kNone).
-                auto issue_qk = [&](const clear_pair_step_t &st, uint32_t keep) {
+                auto issue_qk = [&](const clear_pair_step_t &st) {
                     // the softmax warps must have taken the previous S_t out of tensor memory
                     if (n_qk > 0) ok = wait_bar(b_sfree, (n_qk - 1) & 1u, abort_flag, prm.status, 16);
                     if (!ok) return;
                     const uint32_t pos = ring_base + ((uint32_t)st.load_base & 0xffffu) + (uint32_t)step_tile_index(st.flags, t);
-                    const uint32_t stage = kv_wait(pos, keep);
+                    const uint32_t stage = kv_wait(pos);
                     if (!ok) return;
                     ptx::tc_fence_after();
                     const uint32_t k_lo = ptx::smem_desc_lo(sRing + stage * kTileBytes, 16);
@@ -447,7 +445,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 while (!step_uses(cur.flags, t) && s + 1 < n) cur = load_step(steps + ++s);
                 clear_pair_step_t pre = cur;  // record s + 1, fetched one step ahead
                 if (s + 1 < n) pre = load_step(steps + s + 1);
-                issue_qk(cur, kNone);
+                issue_qk(cur);
                 bool first_pv = true;
                 while (ok) {
                     // next step of this query tile
@@ -470,21 +468,21 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     if (has_next) {
                         const uint32_t pos_k = ring_base + ((uint32_t)nxt.load_base & 0xffffu) + (uint32_t)step_tile_index(nxt.flags, t);
                         if (pos_k < pos_v) {
-                            issue_qk(nxt, kNone);
+                            issue_qk(nxt);
                             qk_done = true;
                             if (!ok) break;
                         }
                     }
 
                     // O_t += P_t V, the two 64-key halves of P one after the other
-                    if (!qk_done) kv_walk(pos_v, kNone);
+                    if (!qk_done) kv_walk(pos_v);
                     uint32_t stage_v = 0;
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         if (h == 0) {
                             ok = wait_bar(ptx::smem_u32(&ctrl->p_ready[t]), n_pv & 1u, abort_flag, prm.status, 7);
                             if (!ok) break;
-                            stage_v = kv_wait(pos_v, kNone);
+                            stage_v = kv_wait(pos_v);
                             if (!ok) break;
                             if (first_pv) {
                                 // the epilogue must have read the previous item's O_t out of tensor memory
@@ -514,13 +512,13 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         ptx::tc_commit(ptx::smem_u32(&ctrl->o_full[t]));
                         break;
                     }
-                    if (!qk_done) issue_qk(nxt, kNone);
+                    if (!qk_done) issue_qk(nxt);
                     cur = nxt;
                     s = s2;
                 }
                 ++n_it;
                 ring_base += (uint32_t)item.n_loads;
-                kv_walk(ring_base, kNone);
+                kv_walk(ring_base);
             }
             if (*abort_flag) {
                 // MMAs that were issued must retire before tensor memory is given back
@@ -545,7 +543,10 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]), b_pready = ptx::smem_u32(&ctrl->p_ready[t]);
         // this row of the two P half-tiles (64 keys each): K-major, 128-byte rows, 16-byte chunks
         // XOR-swizzled by the row number
-        uint8_t *p_row = smem_raw + (sP - smem_base) + t * 2 * kHalfBytes + r * 128;
+        const uint32_t p_row = sP + t * 2 * kHalfBytes + r * 128;
+        uint32_t p_chunk[8];  // where the eight 16-byte chunks of a row go
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) p_chunk[ch] = p_row + (uint32_t)((ch ^ (r & 7)) << 4);
         uint32_t n_s = 0, n_items_seen = 0;
         bool alive = true;
         for (uint32_t k = 0; alive; ++k) {
@@ -737,8 +738,8 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
 #pragma unroll
                         for (int cc = 0; cc < 2; ++cc) {
                             const int ch = 4 * (w & 1) + 2 * grp + cc;  // chunk of the 128-byte row of half w / 2
-                            *reinterpret_cast<uint4 *>(p_row + (w >> 1) * kHalfBytes + ((ch ^ (r & 7)) << 4)) =
-                                make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+                            ptx::st_shared_v4(p_chunk[ch] + (w >> 1) * kHalfBytes, pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2],
+                                              pk[4 * cc + 3]);
                         }
                     }
                 }
