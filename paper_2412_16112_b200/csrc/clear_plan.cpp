@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <map>
 #include <utility>
 
@@ -218,11 +219,15 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
     sch.mask_table.clear();
 
     // Eq. 3 for a key patch at offset (dy, dx) from a query patch, once per distinct offset
+    // (CLEAR_MAX_MASK_ENTRIES lowers the cap of the table; with 0 every masked patch takes the kernel's
+    // table-free path, which is otherwise reached only by very large radii)
+    int max_entries = kMaxMaskEntries;
+    if (const char *e = std::getenv("CLEAR_MAX_MASK_ENTRIES")) max_entries = std::max(0, std::min(kMaxMaskEntries, std::atoi(e)));
     std::map<std::pair<int, int>, int> mask_ids;
     auto mask_entry = [&](int dy, int dx) -> int {
         auto it = mask_ids.find({dy, dx});
         if (it != mask_ids.end()) return it->second;
-        if ((int)mask_ids.size() >= kMaxMaskEntries) return -1;
+        if ((int)mask_ids.size() >= max_entries) return -1;
         const int id = (int)mask_ids.size();
         mask_ids[{dy, dx}] = id;
         sch.mask_table.resize((size_t)(id + 1) * kTileTokens * 4, 0u);

@@ -147,6 +147,19 @@ def test_ws_kernel_many_heads_keep_the_queue_busy():
     assert float((got.float() - other.float()).abs().max()) <= 2e-2
 
 
+@pytest.mark.parametrize("cap", ["0", "2"])
+def test_ws_kernel_without_a_mask_table(cap, monkeypatch):
+    """Patches beyond the mask table's capacity evaluate Eq. 3 from the half-width table in the kernel
+    (normally only very large radii get there): forced here by capping the table."""
+    monkeypatch.setenv("CLEAR_MAX_MASK_ENTRIES", cap)
+    gh, gw, T, r, d = 29, 37, 70, 6.5, 128
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=606)
+    scale = 1 / math.sqrt(d)
+    want = oracle.attn(q, k, v, gh, gw, T, r, scale)
+    got = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_TCGEN05_WS)
+    assert_close_bf16(got, want, f"table cap {cap}")
+
+
 @pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_IDS)
 def test_tc_kernel_split_text_rows_small(kernel):
     """N large enough that the text-query rows are split over key ranges and merged."""

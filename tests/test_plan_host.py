@@ -338,6 +338,23 @@ def test_pair_schedule_covers_each_allowed_pair_exactly_once(gh, gw, T, r):
         assert info.workspace_bytes == len(slots) * 128 * (128 + 2) * 4
 
 
+def test_mask_table_cap_sends_patches_to_the_table_free_path(monkeypatch):
+    monkeypatch.setenv("CLEAR_MAX_MASK_ENTRIES", "3")
+    p = clear.Plan(1, 1, 40, 40, 0, 128, 9.0, kernel=clear.KERNEL_TCGEN05_WS, host_only=True)
+    items, steps = p.pair_tables()
+    assert len(p.mask_table()) == 3
+    ids = set()
+    for it in items:
+        for st in steps[it.step_begin: it.step_begin + it.step_count]:
+            if st.flags & clear.STEP_LINEAR:
+                continue
+            if st.flags & clear.STEP_USE0 and st.flags & clear.STEP_MASKED0:
+                ids.add(st.n_valid0)
+            if st.flags & clear.STEP_USE1 and st.flags & clear.STEP_MASKED1:
+                ids.add(st.n_valid1)
+    assert ids == {-1, 0, 1, 2}
+
+
 def test_pair_schedule_at_the_8k_workload():
     p = clear.Plan(1, 24, 512, 512, 512, 128, 16.0, host_only=True)
     info = p.info()
