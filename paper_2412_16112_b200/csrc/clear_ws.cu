@@ -569,8 +569,8 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
 
-            // The next step's record is fetched at the top of a step and this row's precomputed mask words
-            // for it in the middle, so that neither latency is on the critical path.
+            // Step records are fetched two steps ahead and this row's precomputed mask words one step ahead,
+            // so that neither latency is on the critical path.
             const int kMaskedBit = t ? CLEAR_STEP_MASKED1 : CLEAR_STEP_MASKED0;
             auto load_mask_row = [&](const SideStep &q) -> uint4 {
                 if (step_uses(q.flags, t) && (q.flags & kMaskedBit) && !(q.flags & CLEAR_STEP_LINEAR) && q.n_valid >= 0)
@@ -578,11 +578,14 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 return make_uint4(0u, 0u, 0u, 0u);
             };
             SideStep st_next = load_side_step(steps, t);
+            SideStep st_next2 = st_next;
+            if (step_count > 1) st_next2 = load_side_step(steps + 1, t);
             uint4 mrow_next = load_mask_row(st_next);
             for (int s = 0; s < step_count; ++s) {
                 const SideStep st = st_next;
                 const uint4 mrow = mrow_next;
-                if (s + 1 < step_count) st_next = load_side_step(steps + s + 1, t);
+                st_next = st_next2;  // fetched a step ago: the mask row's address does not wait for it
+                if (s + 2 < step_count) st_next2 = load_side_step(steps + s + 2, t);
                 if (!step_uses(st.flags, t)) {
                     if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
                     continue;
