@@ -200,10 +200,15 @@ int clear_attn_fwd_planned(const clear_plan_t *plan, const void *q, const void *
                            void *out, float scale, void *stream);
 
 /* Forward pass on HOST tensors (same layout and dtype as the plan's): copies q, k, v to staging
- * buffers the plan owns (allocated on first use), runs the kernels, copies `out` back, all on
- * `stream`, and returns after synchronising that stream.  Pinned host memory makes the copies
- * asynchronous with respect to other streams.  Errors as clear_attn_fwd_planned, plus NO_MEMORY
- * and DEVICE_TIMEOUT. */
+ * buffers the plan owns (allocated on first use), runs the kernels, copies `out` back, and returns
+ * after synchronising `stream`.  A problem of more than one chunk (a chunk = whole (b, h) slices of
+ * at least 96 MiB per tensor, at most 16 chunks; the environment variable CLEAR_HOST_CHUNK_BYTES,
+ * read at the plan's first call, changes the size) runs as a three-stage pipeline: the copies in,
+ * the kernels (on `stream`, with a plan per chunk size that this plan owns) and the copies out each
+ * work on a different chunk, on two extra streams the plan creates, so both PCIe directions and
+ * the GPU are busy at once; results are identical to the one-piece run.  Only pinned host memory
+ * lets the stages overlap.  Eq. 1 and Eq. 3 hold per (b, h) slice, so cutting that axis changes
+ * nothing.  Errors as clear_attn_fwd_planned, plus NO_MEMORY and DEVICE_TIMEOUT. */
 int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_host,
                         const void *v_host, void *out_host, float scale, void *stream);
 

@@ -135,6 +135,83 @@ int create_plan(clear_plan_t **out, const Shape &shape_in, bool host_only)
     return CLEAR_OK;
 }
 
+// Chunks of the host-tensor entry point hold at least this many bytes per tensor (CLEAR_HOST_CHUNK_BYTES
+// overrides it): large enough that a chunk's kernels fill the device, small enough that the first
+// copy in and the last copy out, which nothing overlaps, stay short.
+constexpr size_t kHostChunkBytes = (size_t)96 << 20;
+
+void destroy_host_pipe(clear_plan *p)
+{
+    HostPipe *h = p->pipe;
+    if (!h) return;
+    for (clear_plan *&sub : h->sub) {
+        (void)clear_plan_destroy(sub);
+        sub = nullptr;
+    }
+    if (h->s_in) (void)cudaStreamDestroy(h->s_in);
+    if (h->s_out) (void)cudaStreamDestroy(h->s_out);
+    if (h->ev_start) (void)cudaEventDestroy(h->ev_start);
+    if (h->ev_out) (void)cudaEventDestroy(h->ev_out);
+    for (cudaEvent_t ev : h->ev_in)
+        if (ev) (void)cudaEventDestroy(ev);
+    for (cudaEvent_t ev : h->ev_done)
+        if (ev) (void)cudaEventDestroy(ev);
+    (void)cudaGetLastError();
+    delete h;
+    p->pipe = nullptr;
+}
+
+// Builds the copy/compute pipeline of the host-tensor entry point on first use; leaves `plan->pipe`
+// null when the problem is too small to be worth cutting.  `slice` = bytes of one (b, h) slice.
+int ensure_host_pipe(clear_plan *plan, size_t slice)
+{
+    if (plan->pipe || plan->pipe_decided) return CLEAR_OK;
+    plan->pipe_decided = true;
+    const Shape &s = plan->shape;
+    const int n_bh = s.B * s.H;
+    size_t min_bytes = kHostChunkBytes;
+    if (const char *e = std::getenv("CLEAR_HOST_CHUNK_BYTES")) min_bytes = (size_t)std::max(1ll, std::atoll(e));
+    int chunk = (int)std::min<size_t>((size_t)n_bh, (min_bytes + slice - 1) / slice);
+    chunk = std::max(chunk, (n_bh + kMaxHostChunks - 1) / kMaxHostChunks);
+    if (chunk >= n_bh) return CLEAR_OK;
+    std::unique_ptr<HostPipe> hp(new (std::nothrow) HostPipe());
+    if (!hp) return CLEAR_ERR_NO_MEMORY;
+    hp->chunk_heads = chunk;
+    hp->n_chunks = (n_bh + chunk - 1) / chunk;
+    plan->pipe = hp.release();
+    HostPipe &h = *plan->pipe;
+    auto fail = [&](int rc) {
+        destroy_host_pipe(plan);
+        plan->pipe_decided = false;
+        return rc;
+    };
+    Shape sub = s;
+    sub.kernel = plan->kernel;
+    sub.B = 1;
+    sub.H = chunk;
+    int rc = create_plan(&h.sub[0], sub, false);
+    if (rc != CLEAR_OK) return fail(rc);
+    if (n_bh % chunk) {
+        sub.H = n_bh % chunk;
+        rc = create_plan(&h.sub[1], sub, false);
+        if (rc != CLEAR_OK) return fail(rc);
+    }
+    cudaError_t e = cudaStreamCreateWithFlags(&h.s_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h.s_out, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h.ev_start, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h.ev_out, cudaEventDisableTiming);
+    for (int c = 0; c < h.n_chunks && e == cudaSuccess; ++c) {
+        e = cudaEventCreateWithFlags(&h.ev_in[c], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h.ev_done[c], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) {
+        note_cuda_error((int)e);
+        (void)cudaGetLastError();
+        return fail(CLEAR_ERR_CUDA);
+    }
+    return CLEAR_OK;
+}
+
 int check_tensors(const void *q, const void *k, const void *v, const void *out)
 {
     if (!q || !k || !v || !out) return CLEAR_ERR_INVALID_ARG;
@@ -282,7 +359,8 @@ int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_ho
     if (dev != plan->device) return CLEAR_ERR_PLAN_MISMATCH;
     const Shape &s = plan->shape;
     const size_t esz = s.dtype == CLEAR_BF16 ? 2 : 4;
-    const size_t bytes = (size_t)s.B * s.H * ((size_t)s.n_text + (size_t)s.grid_h * s.grid_w) * s.head_dim * esz;
+    const size_t slice = ((size_t)s.n_text + (size_t)s.grid_h * s.grid_w) * s.head_dim * esz;
+    const size_t bytes = (size_t)s.B * s.H * slice;
     for (void *&st : plan->d_stage) {
         if (!st) {
             cudaError_t e = cudaMalloc(&st, bytes);
@@ -295,13 +373,62 @@ int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_ho
         }
     }
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[0], q_host, bytes, cudaMemcpyHostToDevice, cs));
-    CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[1], k_host, bytes, cudaMemcpyHostToDevice, cs));
-    CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[2], v_host, bytes, cudaMemcpyHostToDevice, cs));
-    int rc = forward(plan, plan->d_stage[0], plan->d_stage[1], plan->d_stage[2], plan->d_stage[3], scale, stream);
+    int rc = ensure_host_pipe(plan, slice);
     if (rc != CLEAR_OK) return rc;
-    CLEAR_CUDA_TRY(cudaMemcpyAsync(out_host, plan->d_stage[3], bytes, cudaMemcpyDeviceToHost, cs));
-    return clear_plan_check(plan, stream);
+    if (!plan->pipe) {
+        CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[0], q_host, bytes, cudaMemcpyHostToDevice, cs));
+        CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[1], k_host, bytes, cudaMemcpyHostToDevice, cs));
+        CLEAR_CUDA_TRY(cudaMemcpyAsync(plan->d_stage[2], v_host, bytes, cudaMemcpyHostToDevice, cs));
+        rc = forward(plan, plan->d_stage[0], plan->d_stage[1], plan->d_stage[2], plan->d_stage[3], scale, stream);
+        if (rc != CLEAR_OK) return rc;
+        CLEAR_CUDA_TRY(cudaMemcpyAsync(out_host, plan->d_stage[3], bytes, cudaMemcpyDeviceToHost, cs));
+        return clear_plan_check(plan, stream);
+    }
+
+    // Three stages over chunks of the (batch, head) axis: copies in on one stream, kernels on the
+    // caller's stream, copies out on a third; events hand each chunk from stage to stage.
+    HostPipe &hp = *plan->pipe;
+    const int n_bh = s.B * s.H;
+    const void *host_in[3] = {q_host, k_host, v_host};
+    CLEAR_CUDA_TRY(cudaEventRecord(hp.ev_start, cs));
+    CLEAR_CUDA_TRY(cudaStreamWaitEvent(hp.s_in, hp.ev_start, 0));
+    CLEAR_CUDA_TRY(cudaStreamWaitEvent(hp.s_out, hp.ev_start, 0));
+    rc = CLEAR_OK;
+    for (int c = 0; c < hp.n_chunks && rc == CLEAR_OK; ++c) {
+        const int first = c * hp.chunk_heads;
+        const int heads = std::min(hp.chunk_heads, n_bh - first);
+        const size_t off = (size_t)first * slice, len = (size_t)heads * slice;
+        for (int t = 0; t < 3; ++t)
+            CLEAR_CUDA_TRY(cudaMemcpyAsync((char *)plan->d_stage[t] + off, (const char *)host_in[t] + off, len,
+                                           cudaMemcpyHostToDevice, hp.s_in));
+        CLEAR_CUDA_TRY(cudaEventRecord(hp.ev_in[c], hp.s_in));
+        CLEAR_CUDA_TRY(cudaStreamWaitEvent(cs, hp.ev_in[c], 0));
+        const clear_plan *sub = heads == hp.chunk_heads ? hp.sub[0] : hp.sub[1];
+        rc = forward(sub, (char *)plan->d_stage[0] + off, (char *)plan->d_stage[1] + off,
+                     (char *)plan->d_stage[2] + off, (char *)plan->d_stage[3] + off, scale, stream);
+        if (rc != CLEAR_OK) break;
+        CLEAR_CUDA_TRY(cudaEventRecord(hp.ev_done[c], cs));
+        CLEAR_CUDA_TRY(cudaStreamWaitEvent(hp.s_out, hp.ev_done[c], 0));
+        CLEAR_CUDA_TRY(cudaMemcpyAsync((char *)out_host + off, (char *)plan->d_stage[3] + off, len,
+                                       cudaMemcpyDeviceToHost, hp.s_out));
+    }
+    // the copies out are joined back into the caller's stream, error or not (the copies in already
+    // are: every chunk's kernels waited for them)
+    cudaError_t e1 = cudaEventRecord(hp.ev_out, hp.s_out);
+    cudaError_t e2 = cudaStreamWaitEvent(cs, hp.ev_out, 0);
+    for (cudaError_t e : {e1, e2})
+        if (e != cudaSuccess) {
+            note_cuda_error((int)e);
+            (void)cudaGetLastError();
+            if (rc == CLEAR_OK) rc = CLEAR_ERR_CUDA;
+        }
+    for (clear_plan *sub : hp.sub)
+        if (sub) {
+            const int r = clear_plan_check(sub, stream);
+            if (rc == CLEAR_OK) rc = r;
+        }
+    if (rc != CLEAR_OK) (void)cudaStreamSynchronize(cs);
+    return rc;
 }
 
 int clear_plan_info(const clear_plan_t *plan, clear_plan_info_t *info)
@@ -357,6 +484,7 @@ int clear_plan_destroy(clear_plan_t *plan)
     if (!plan->host_only) {
         int prev = -1;
         if (cudaGetDevice(&prev) == cudaSuccess && prev != plan->device) (void)cudaSetDevice(plan->device);
+        destroy_host_pipe(plan);
         rc = free_device_parts(plan);
         if (prev >= 0 && prev != plan->device) (void)cudaSetDevice(prev);
     }

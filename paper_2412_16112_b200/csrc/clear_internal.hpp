@@ -8,6 +8,24 @@
 #include "clear_attn.h"
 #include "clear_plan.hpp"
 
+namespace clear {
+
+// The host-tensor entry point cuts the (batch, head) axis into chunks: while chunk c is computed,
+// chunk c+1 travels to the device and chunk c-1 travels back.  Each chunk size has a plan of its own
+// (B = 1, H = heads of the chunk); streams and events order the three stages.
+constexpr int kMaxHostChunks = 16;
+struct HostPipe {
+    int chunk_heads = 0;              // (b, h) slices per full chunk
+    int n_chunks = 0;
+    clear_plan *sub[2] = {nullptr, nullptr};  // plan of a full chunk, plan of the shorter last chunk
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr;
+    cudaEvent_t ev_in[kMaxHostChunks] = {};
+    cudaEvent_t ev_done[kMaxHostChunks] = {};
+};
+
+}  // namespace clear
+
 struct clear_plan {
     clear::Shape shape;
     clear::Schedule sch;
@@ -35,6 +53,10 @@ struct clear_plan {
 
     // staging buffers of the host-tensor entry point (owned, allocated on first use)
     void *d_stage[4] = {nullptr, nullptr, nullptr, nullptr};
+    // copy/compute pipeline of the host-tensor entry point (owned, built on first use; null while
+    // the whole problem goes through in one piece)
+    clear::HostPipe *pipe = nullptr;
+    bool pipe_decided = false;
 
     // tensor maps of the last (q, k, v, out) seen by the tensor-core launcher
     mutable std::mutex tm_mutex;

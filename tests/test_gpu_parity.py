@@ -365,3 +365,29 @@ def test_host_tensor_entry_point():
     want = oracle.attn(q, k, v, gh, gw, T, r, scale)
     assert_close_bf16(oh, want, "host entry point")
     plan.destroy()
+
+
+@pytest.mark.parametrize("B,H", [(1, 5), (2, 3)])
+def test_host_tensor_entry_point_in_chunks(B, H, monkeypatch):
+    """With a small chunk size the host path cuts the (batch, head) axis into pieces (two slices per
+    chunk here, so B*H = 5 leaves a shorter last chunk) and overlaps their copies with the kernels;
+    the result must equal, bit for bit, the one-piece run on device tensors, twice in a row."""
+    gh, gw, T, r, d = 24, 32, 150, 5.0, 128
+    q, k, v = workloads.make_custom(B, H, gh, gw, T, d, seed=47)
+    scale = 1 / math.sqrt(d)
+    slice_bytes = (T + gh * gw) * d * 2
+    monkeypatch.setenv("CLEAR_HOST_CHUNK_BYTES", str(2 * slice_bytes))
+    plan = clear.Plan(B, H, gh, gw, T, d, r)
+    qh, kh, vh = (t.pin_memory() for t in (q, k, v))
+    ref = run_plan(q, k, v, gh, gw, T, r, scale, clear.KERNEL_AUTO)
+    for rep in range(2):
+        oh = torch.full_like(q, float("nan")).pin_memory()
+        plan.forward_host(qh, kh, vh, oh, scale)
+        assert torch.equal(oh.view(torch.int16), ref.view(torch.int16)), f"chunked host run {rep} differs"
+    # pageable host memory takes the same route
+    oh = torch.full_like(q, float("nan"))
+    plan.forward_host(q, k, v, oh, scale)
+    assert torch.equal(oh.view(torch.int16), ref.view(torch.int16))
+    want = oracle.attn(q[:1, :2], k[:1, :2], v[:1, :2], gh, gw, T, r, scale)
+    assert_close_bf16(oh[:1, :2], want, "chunked host entry point")
+    plan.destroy()
