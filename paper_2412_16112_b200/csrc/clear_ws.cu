@@ -44,6 +44,13 @@ constexpr uint32_t kSchedReaders = 10;
 // registers per thread of each role: 128 x 64 + 256 x 216 = 63488, within what the block is launched with
 // (384 threads x 168); raising a warp's budget only draws on registers other warps of the block gave back
 constexpr uint32_t kRegsControl = 64, kRegsSoftmax = 216;
+// Left alone, the two query tiles of a pair run their steps in lockstep: both in the exponential phase
+// (special-function unit saturated, tensor core waiting for P), then both waiting for P V.  Tile 1
+// enters an exponential phase this many clocks late whenever a run of steps on a shared key tile begins
+// (the item's first step, and the first shared step after steps in which the tiles read different key
+// tiles and drift back into lockstep waiting for the ring), so that the phases of the two tiles
+// interleave for part of the item (measured: 1.5 to 5 % per call, best near 1200).
+constexpr long long kStaggerClocks = 1200;
 
 struct WsParams {
     const clear_pair_item_t *items;
@@ -568,6 +575,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             const bool q_valid = is_text ? r < (t ? item.n_rows1 : item.n_rows0) : (q_y < prm.grid_h && q_x < prm.grid_w);
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
+            bool prev_shared = false;
 
             // Step records are fetched two steps ahead and this row's precomputed mask words one step ahead,
             // so that neither latency is on the critical path.
@@ -716,6 +724,15 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                         ptx::tmem_wait_st();
                         ptx::tc_fence_before();
                     }
+                }
+                {
+                    const bool shared = (st.flags & CLEAR_STEP_SHARED) != 0;
+                    if (t == 1 && shared && !prev_shared) {
+                        const long long t0 = clock64();
+                        while (clock64() - t0 < kStaggerClocks) {
+                        }
+                    }
+                    prev_shared = shared;
                 }
                 const float mc = (m_used == -INFINITY) ? 0.f : m_used * c;
 
