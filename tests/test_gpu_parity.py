@@ -367,6 +367,42 @@ def test_host_tensor_entry_point():
     plan.destroy()
 
 
+def test_host_tensor_entry_point_in_chunks_at_2048px(monkeypatch):
+    """The 2048px workload through the host path in chunks of at least 40 MiB per tensor (24 heads of 4.3 MB:
+    two chunks of ten heads and a last chunk of four) equals the one-piece run on device tensors bit for bit."""
+    w = workloads.WORKLOADS["c2_2048px_r16"]
+    q, k, v = workloads.make_inputs(w)
+    monkeypatch.setenv("CLEAR_HOST_CHUNK_BYTES", str(40 << 20))
+    plan = clear.Plan(w.B, w.H, w.grid_h, w.grid_w, w.n_text, w.head_dim, w.radius)
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    ref = torch.full_like(qd, float("nan"))
+    plan.forward(qd, kd, vd, ref, w.scale)
+    plan.check()
+    qh, kh, vh = (t.pin_memory() for t in (q, k, v))
+    oh = torch.full_like(q, float("nan")).pin_memory()
+    plan.forward_host(qh, kh, vh, oh, w.scale)
+    assert torch.equal(oh.view(torch.int16), ref.cpu().view(torch.int16))
+    plan.destroy()
+
+
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_IDS)
+def test_transposing_the_grid_permutes_the_outputs_on_the_gpu(kernel):
+    """Eq. 3 depends on the grid offset only through dx^2 + dy^2, so transposing the latent grid (with q, k, v
+    re-ordered to match) must permute the image rows of the output and leave the text rows alone.  The two runs
+    cut the grid into different patches and border shapes: a property that needs no oracle and holds at any size."""
+    gh, gw, T, r, d = 56, 40, 70, 6.0, 128
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=23)
+    scale = 1 / math.sqrt(d)
+    n = gh * gw
+    perm = torch.arange(n).reshape(gh, gw).T.reshape(-1)  # token order of the transposed grid
+    idx = torch.cat([torch.arange(T), T + perm])
+    out = run_plan(q, k, v, gh, gw, T, r, scale, kernel)
+    out_t = run_plan(q[:, :, idx].contiguous(), k[:, :, idx].contiguous(), v[:, :, idx].contiguous(), gw, gh, T, r, scale, kernel)
+    err = (out_t.double() - out[:, :, idx].double()).abs()
+    assert torch.isfinite(err).all()
+    assert err.max().item() <= BF16_MAX and err.mean().item() <= BF16_MEAN, (err.max().item(), err.mean().item())
+
+
 @pytest.mark.parametrize("B,H", [(1, 5), (2, 3)])
 def test_host_tensor_entry_point_in_chunks(B, H, monkeypatch):
     """With a small chunk size the host path cuts the (batch, head) axis into pieces (two slices per
