@@ -123,11 +123,10 @@ typedef struct clear_pair_step {
     int32_t flags;      /* CLEAR_STEP_* bits                                                        */
     int32_t n_valid0;   /* linear tiles: keys [0, n_valid) of the tile exist / are allowed; 2-D patches: */
     int32_t n_valid1;   /*   index of the tile pair's entry in the mask table, or -1 if it has none      */
-    int32_t load_base;  /* where this step's tiles sit in the item's staging order, which runs K(step 0),
-                           then for every step s: K(step s + 1), V(step s) -- K tiles are staged one step
-                           ahead of V tiles.  Low 16 bits: position of the step's first K tile; high 16
-                           bits: position of its first V tile (a step with two distinct key tiles takes
-                           two consecutive positions each time, tile 0's first).                        */
+    int32_t load_base;  /* where this step's tiles sit in the item's staging order, which runs, for every
+                           step in turn, its K tiles and then its V tiles.  Low 16 bits: position of the
+                           step's first K tile; high 16 bits: position of its first V tile (a step with two
+                           distinct key tiles takes two consecutive positions each time, tile 0's first). */
 } clear_pair_step_t;
 
 /* One unit of work of the TCGEN05_WS kernel: two 128-query tiles walking one step list. */

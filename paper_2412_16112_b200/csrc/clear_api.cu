@@ -73,7 +73,7 @@ int create_plan(clear_plan_t **out, const Shape &shape_in, bool host_only)
     Shape s = shape_in;
     int rc = validate_shape(s);
     if (rc != CLEAR_OK) return rc;
-    const int kernel = select_kernel(s);
+    int kernel = select_kernel(s);
     {
         Shape chk = s;
         chk.kernel = kernel;
@@ -83,18 +83,28 @@ int create_plan(clear_plan_t **out, const Shape &shape_in, bool host_only)
     std::unique_ptr<clear_plan> p(new (std::nothrow) clear_plan());
     if (!p) return CLEAR_ERR_NO_MEMORY;
     p->shape = s;
-    p->kernel = kernel;
     p->host_only = host_only;
     try {
+        if (kernel == CLEAR_KERNEL_TCGEN05_WS) {
+            build_pair_schedule(s, p->sch);
+            // An item whose key-tile list outgrows the 16-bit ring positions of the step records (radii of
+            // about a thousand tokens on grids of millions) cannot run on this kernel, and tile lists of
+            // that length would take gigabytes: the CUDA-core kernel, which walks Eq. 3 without any list,
+            // takes over when the choice was left to the library.
+            if (p->sch.pair_overflow) {
+                if (s.kernel != CLEAR_KERNEL_AUTO) return CLEAR_ERR_UNSUPPORTED;
+                kernel = CLEAR_KERNEL_SIMT;
+                p->sch = Schedule();
+            }
+        }
         if (kernel == CLEAR_KERNEL_TCGEN05)
             build_tile_schedule(s, p->sch);
-        else if (kernel == CLEAR_KERNEL_TCGEN05_WS)
-            build_pair_schedule(s, p->sch);
-        else
+        else if (kernel == CLEAR_KERNEL_SIMT)
             build_geometry(s, p->sch);
     } catch (const std::bad_alloc &) {
         return CLEAR_ERR_NO_MEMORY;
     }
+    p->kernel = kernel;
     if (kernel != CLEAR_KERNEL_SIMT && p->sch.n_partial_slots > 0) {
         const int64_t rows = (int64_t)s.B * s.H * p->sch.n_partial_slots * kTileTokens;
         p->workspace_bytes = rows * (s.head_dim + 2) * (int64_t)sizeof(float);

@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <climits>
 #include <cstdlib>
 #include <map>
 #include <utility>
@@ -217,6 +218,7 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
     sch.pair_items.clear();
     sch.pair_steps.clear();
     sch.mask_table.clear();
+    sch.pair_overflow = false;
 
     // Eq. 3 for a key patch at offset (dy, dx) from a query patch, once per distinct offset
     // (CLEAR_MAX_MASK_ENTRIES lowers the cap of the table; with 0 every masked patch takes the kernel's
@@ -243,7 +245,7 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
     };
 
     auto finish_item = [&](clear_pair_item_t &it) {
-        // staging order: K(0), then K(s + 1), V(s) for every step s (K runs one step ahead of V)
+        // staging order: for every step its K tiles, then its V tiles (the order the MMAs read them in)
         auto n_tiles = [&](int32_t i) {
             const clear_pair_step_t &st = sch.pair_steps[(size_t)i];
             const int a = (st.flags & CLEAR_STEP_USE0) ? 1 : 0;
@@ -251,20 +253,16 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
             return a + b;
         };
         const int32_t first = it.step_begin, end = (int32_t)sch.pair_steps.size();
-        int32_t pos = 0;
-        std::vector<int32_t> k_pos((size_t)(end - first), 0);
-        k_pos[0] = pos;
-        pos += n_tiles(first);
+        int64_t pos = 0;
         for (int32_t i = first; i < end; ++i) {
-            if (i + 1 < end) {
-                k_pos[(size_t)(i + 1 - first)] = pos;
-                pos += n_tiles(i + 1);
-            }
-            sch.pair_steps[(size_t)i].load_base = k_pos[(size_t)(i - first)] | (pos << 16);
-            pos += n_tiles(i);
+            const int64_t k_pos = pos, v_pos = pos + n_tiles(i);
+            pos = v_pos + n_tiles(i);
+            // positions travel in 16 bits each
+            if (pos > 0xffff) sch.pair_overflow = true;
+            sch.pair_steps[(size_t)i].load_base = (int32_t)((k_pos & 0xffff) | ((v_pos & 0xffff) << 16));
         }
         it.step_count = end - first;
-        it.n_loads = pos;
+        it.n_loads = (int32_t)std::min<int64_t>(pos, INT_MAX);
         sch.pair_items.push_back(it);
     };
     auto linear_step = [&](int x, int n_valid, int n_sides) {
@@ -382,6 +380,9 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
                 sch.pair_steps.push_back(st);
             }
             finish_item(it);
+            // a list too long for the step records' 16-bit ring positions: this kernel cannot run the
+            // shape, and the remaining lists (gigabytes at such radii) are not worth building
+            if (sch.pair_overflow) return;
         }
     }
 

@@ -34,6 +34,7 @@ struct Schedule {
     std::vector<clear_pair_item_t> pair_items;   // TCGEN05_WS: text items first, then image items
     std::vector<clear_pair_step_t> pair_steps;
     int n_text_pair_items = 0;
+    bool pair_overflow = false;                  // an item stages more tiles than its 16-bit positions can name
     std::vector<uint32_t> mask_table;            // TCGEN05_WS: [entry][128 query rows][4 words]
     int n_text_tiles = 0;                // text-query tiles of 128 rows
     int n_text_splits = 0;               // splits per text-query tile (1 = no partial results)

@@ -7,23 +7,26 @@
 //
 // Roles (384 threads):
 //   warp 0        : takes items from the queue and issues every TMA load (Q tiles, K/V ring);
-//   warps 1, 2    : one thread each issues the tcgen05.mma of query tile t = 0, 1: S_t = Q_t K^T,
-//                   O_t += P_t V; the softmax of one query tile runs under the MMAs of the other;
+//   warp 1        : one thread issues every tcgen05.mma, alternating between the two query tiles:
+//                   S_t = Q_t K^T, O_t += P_t V; the softmax of one tile runs under the MMAs of the other;
 //   warps 4-7     : softmax and epilogue of query tile 0 (thread r owns query row r = tensor-memory
-//                   lane r): mask, running maximum, P = exp2(.) as bf16 into shared memory, row sum; at the
-//                   end of an item O / l -> bf16 -> global memory (or fp32 partial results of split text
-//                   rows);
+//                   lane r): running maximum, P = exp2(.) on the keys Eq. 3 allows and 0 elsewhere, as
+//                   bf16 into tensor memory over S, row sum; at the end of an item O / l -> bf16 ->
+//                   global memory (or fp32 partial results of split text rows);
 //   warps 8-11    : the same for query tile 1.
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each.  P goes through shared memory, so
-// that S_t of the next step can be computed while the softmax of this one runs.
-// Shared memory: Q0, Q1, a ring of three key/value stages (K and V tiles take one stage each) and P
-// of each query tile.
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each; P_t takes the first 64 columns of
+// S_t and is the tensor-memory operand of P_t V, so that P never crosses shared memory: with both MMA
+// operands in shared memory a 128 x 128 x 16 MMA reads 8 KB per 64 clocks, all a shared memory can
+// deliver, and nothing else (P stores, TMA fills) fits beside it.
+// Shared memory: Q0, Q1 and a ring of five key/value stages (K and V tiles take one stage each).
 // Every wait is bounded: on expiry the block raises the plan's status word and leaves.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstdio>
 #include <cstring>
+#include <type_traits>
 
 #include "clear_internal.hpp"
 #include "ptx.cuh"
@@ -32,25 +35,30 @@ namespace clear {
 namespace {
 
 constexpr int kWsThreads = 384;   // 4 control warps + 2 x 4 softmax warps
-constexpr int kRing = 3;
+constexpr int kRing = 5;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr uint32_t kWaitHintNs = 20000;            // one sleep inside try_wait
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
 constexpr float kRescaleThreshold = 8.f;  // log2 units: O is rescaled only when the row max grows by more
+constexpr float kMaxTileSum = 256.f;      // 2^kRescaleThreshold: a row sum of P up to this needs no look at the maximum
 constexpr int kSchedDepth = 2;
-// arrivals that free a queue slot: the two MMA threads and one lane of each of the 8 softmax warps
-constexpr uint32_t kSchedReaders = 10;
-// registers per thread of each role: 128 x 64 + 256 x 216 = 63488, within what the block is launched with
+// arrivals that free a queue slot: the MMA thread and one lane of each of the 8 softmax warps
+constexpr uint32_t kSchedReaders = 9;
+// registers per thread of each role: 128 x 80 + 256 x 208 = 63488, within what the block is launched with
 // (384 threads x 168); raising a warp's budget only draws on registers other warps of the block gave back
-constexpr uint32_t kRegsControl = 64, kRegsSoftmax = 216;
-// Left alone, the two query tiles of a pair run their steps in lockstep: both in the exponential phase
-// (special-function unit saturated, tensor core waiting for P), then both waiting for P V.  Tile 1
-// enters an exponential phase this many clocks late whenever a run of steps on a shared key tile begins
-// (the item's first step, and the first shared step after steps in which the tiles read different key
-// tiles and drift back into lockstep waiting for the ring), so that the phases of the two tiles
-// interleave for part of the item (measured: 1.5 to 5 % per call, best near 1200).
-constexpr long long kStaggerClocks = 1200;
+constexpr uint32_t kRegsControl = 80, kRegsSoftmax = 208;
+static_assert(128 * kRegsControl + 256 * kRegsSoftmax <= 384 * 168, "a raise beyond the block's registers would wait for ever");
+
+// Optional timeline of the softmax warps (compile with -DCLEAR_WS_TRACE): clocks per phase, summed over the
+// launch, printed by block 0.  Off in the product build.
+#ifdef CLEAR_WS_TRACE
+#define TRACE_DECL unsigned long long tr_acc[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; long long tr_t = clock64(); unsigned tr_steps = 0;
+#define TRACE_MARK(i) { const long long tr_n = clock64(); tr_acc[i] += (unsigned long long)(tr_n - tr_t); tr_t = tr_n; }
+#else
+#define TRACE_DECL
+#define TRACE_MARK(i)
+#endif
 
 struct WsParams {
     const clear_pair_item_t *items;
@@ -72,9 +80,9 @@ struct WsParams {
 struct Ctrl {
     uint64_t q_full[2], q_empty[2];
     uint64_t kv_full[kRing], kv_empty[kRing];
-    uint64_t s_full[2], s_free[2], p_ready[2], p_free[2], o_full[2], o_empty[2];
+    uint64_t s_full[2], p_ready[2], o_full[2], o_empty[2];
     uint64_t sched_full[kSchedDepth], sched_empty[kSchedDepth];
-    uint64_t drain[2];
+    uint64_t drain[1];
     int32_t sched_item[kSchedDepth];            // queue position, >= total: no more work
     int32_t sched_bh[kSchedDepth];
     clear_pair_item_t sched_rec[kSchedDepth];   // the item's record, read once from global memory
@@ -208,9 +216,9 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t smem_base = ptx::smem_u32(smem_raw);
-    // Q0, Q1 | ring of K/V stages | P of each query tile as two half-tiles (128 queries x 64 keys) | control
-    const uint32_t sQ = smem_base, sRing = sQ + 2 * kTileBytes, sP = sRing + kRing * kTileBytes;
-    constexpr uint32_t kCtrlOff = (2 + kRing) * kTileBytes + 4 * kHalfBytes;
+    // Q0, Q1 | ring of K/V stages | control
+    const uint32_t sQ = smem_base, sRing = sQ + 2 * kTileBytes;
+    constexpr uint32_t kCtrlOff = (2 + kRing) * kTileBytes;
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_raw + kCtrlOff);
     volatile int *abort_flag = &ctrl->abort_flag;
 
@@ -246,22 +254,19 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->q_empty[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->s_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->s_free[i]), 4);  // one arrival per softmax warp of the tile
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i]), 4);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->p_free[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->p_ready[i]), 4);  // one arrival per softmax warp of the tile
             ptx::mbar_init(ptx::smem_u32(&ctrl->o_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->o_empty[i]), 4);
         }
         for (int i = 0; i < kRing; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->kv_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctrl->kv_empty[i]), 2);
+            ptx::mbar_init(ptx::smem_u32(&ctrl->kv_empty[i]), 1);
         }
         for (int i = 0; i < kSchedDepth; ++i) {
             ptx::mbar_init(ptx::smem_u32(&ctrl->sched_full[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctrl->sched_empty[i]), kSchedReaders);
         }
         ptx::mbar_init(ptx::smem_u32(&ctrl->drain[0]), 1);
-        ptx::mbar_init(ptx::smem_u32(&ctrl->drain[1]), 1);
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
@@ -310,8 +315,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     }
                     ++n_q[t];
                 }
-                // K/V stages in the plan's staging order: K(step 0), then K(step s + 1), V(step s) for every
-                // step s, so that a step's K tile is on its way a whole step before its V tile is needed
+                // K/V stages in the plan's staging order: for every step its K tiles, then its V tiles
                 auto stage_tiles = [&](const clear_pair_step_t &st, int kv) {
                     const bool has_a = (st.flags & CLEAR_STEP_USE0) != 0;
                     const bool has_b = (st.flags & CLEAR_STEP_USE1) && !(st.flags & CLEAR_STEP_SHARED);
@@ -338,17 +342,13 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 };
                 const clear_pair_step_t *steps = prm.steps + item.step_begin;
                 clear_pair_step_t st = load_step(steps);
-                clear_pair_step_t st_next = st;
-                if (item.step_count > 1) st_next = load_step(steps + 1);
-                stage_tiles(st, 0);
                 for (int s = 0; s < item.step_count && ok; ++s) {
                     // records are fetched ahead of their use, so their latency is off the critical path
-                    clear_pair_step_t st_next2 = st_next;
-                    if (s + 2 < item.step_count) st_next2 = load_step(steps + s + 2);
-                    if (s + 1 < item.step_count) stage_tiles(st_next, 0);
+                    clear_pair_step_t st_next = st;
+                    if (s + 1 < item.step_count) st_next = load_step(steps + s + 1);
+                    stage_tiles(st, 0);
                     stage_tiles(st, 1);
                     st = st_next;
-                    st_next = st_next2;
                 }
                 if (!ok) break;
             }
@@ -361,199 +361,167 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     drain_bar(ptx::smem_u32(&ctrl->kv_full[idx % kRing]), (idx / kRing) & 1u);
                 }
             }
-        } else if ((warp == 1 || warp == 2) && lane == 0) {
-            // ================= MMA issuer of query tile t: S_t = Q_t K^T, O_t += P_t V ===============
-            // One thread per query tile, so that neither tile waits for the other's softmax; the
-            // tensor core runs each thread's MMAs in the order that thread issued them.
-            // S_t(next) is issued as soon as the softmax warps have taken S_t into registers, i.e.
-            // before P_t V of the current step: P travels through shared memory, in two halves of 64 keys.
-            const int t = warp - 1;
+        } else if (warp == 1) {
+            // ================= MMA issuer: S_t = Q_t K^T, O_t += P_t V for both query tiles ============
+            // One thread issues for both tiles in a fixed order -- at every step, for t = 0, 1:
+            // P_t V of tile t's previous step (as soon as its softmax warps have put P_t into tensor
+            // memory), then S_t = Q_t K^T of this step, which overwrites P_t only after P_t V has read it
+            // (same issue order, same pipe).  The tensor core runs the groups in that order, so S_0 is
+            // ready half a step before S_1, the two softmax phases settle half a step apart, and each
+            // tile's exponentials run under the other tile's MMAs.
+            // The whole warp walks the loop in step and one elected lane issues: with warp-uniform control
+            // flow and values the descriptor arithmetic stays on the uniform datapath, and an MMA costs few
+            // enough issue slots to keep the tensor core fed while the softmax warps of the same scheduler
+            // are in their exponential phase (a lone thread in a divergent branch could not: 96 clocks per
+            // MMA against 64 of execution).
             constexpr uint32_t kDescHiK = ptx::smem_desc_hi_sw128(1024);  // 8-row groups are 1024 bytes apart
-            const uint32_t q_lo = ptx::smem_desc_lo(sQ + t * kTileBytes, 16);
-            const uint32_t p_lo = ptx::smem_desc_lo(sP + t * 2 * kHalfBytes, 16);
-            const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
-            const uint32_t b_sfull = ptx::smem_u32(&ctrl->s_full[t]), b_sfree = ptx::smem_u32(&ctrl->s_free[t]);
-            const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]);
+            auto uni = [](int v) { return __shfl_sync(0xffffffffu, v, 0); };  // tells the compiler v is warp-uniform
             uint32_t ring_base = 0;  // K/V stages filled by the items before this one
-            uint32_t n_it = 0;       // items in which this query tile existed
-            uint32_t n_qk = 0;       // S tiles issued
-            uint32_t n_pv = 0;       // steps whose P V has been issued
+            uint32_t n_it[2] = {0, 0};   // items in which the query tile existed
+            uint32_t n_pv[2] = {0, 0};   // steps whose P V has been issued
             bool ok = true;
-            // Both MMA threads walk EVERY ring position in order and arrive once on its "empty" barrier: with
-            // an MMA commit where they read the stage, at once where they do not.  A stage is refilled only
-            // after both arrivals, so neither thread ever waits on a barrier phase that is more than one
-            // ahead of the barrier (mbarrier waits tell phases apart by one parity bit only).
-            uint32_t next_pos = 0;  // first position whose fill this thread has not seen yet
-            // see the fills of [next_pos, pos), stages this thread does not read, and free them at once
-            auto kv_walk = [&](uint32_t pos) {
-                for (; next_pos < pos && ok; ++next_pos) {
-                    const uint32_t st = next_pos % kRing, fl = next_pos / kRing;
-                    ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[st]), fl & 1u, abort_flag, prm.status, 15);
-                    if (ok) ptx::mbar_arrive(ptx::smem_u32(&ctrl->kv_empty[st]));
-                }
+            TRACE_DECL
+            // Every staged tile is read by this warp: it waits once for the fill of a ring position and
+            // frees the stage with an MMA commit behind the last MMA that reads it (a key tile both query
+            // tiles share is read by tile 0 first and freed behind tile 1's MMA).
+            auto kv_wait = [&](uint32_t pos) {
+                if (ok)
+                    ok = __all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->kv_full[pos % kRing]), (pos / kRing) & 1u, abort_flag, prm.status, 4));
             };
-            // wait for the fill of `pos`, a stage this thread reads
-            auto kv_wait = [&](uint32_t pos) -> uint32_t {
-                kv_walk(pos);
-                const uint32_t stage = pos % kRing, fill = pos / kRing;
-                if (ok && next_pos == pos) {
-                    ok = wait_bar(ptx::smem_u32(&ctrl->kv_full[stage]), fill & 1u, abort_flag, prm.status, 4);
-                    next_pos = pos + 1;
-                }
-                return stage;
-            };
-            auto kv_release = [&](uint32_t stage) { ptx::tc_commit(ptx::smem_u32(&ctrl->kv_empty[stage])); };
             for (uint32_t k = 0; ok; ++k) {
                 const uint32_t slot = k % kSchedDepth, use = k / kSchedDepth;
-                if (!wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 5)) break;
-                const int g = ctrl->sched_item[slot];
-                const clear_pair_item_t item = ctrl->sched_rec[slot];
-                ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
+                if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->sched_full[slot]), use & 1u, abort_flag, prm.status, 5))) break;
+                const int g = uni(ctrl->sched_item[slot]);
+                const int n_sides = uni(ctrl->sched_rec[slot].n_sides);
+                const int step_begin = uni(ctrl->sched_rec[slot].step_begin);
+                const int n = uni(ctrl->sched_rec[slot].step_count);
+                const int n_loads = uni(ctrl->sched_rec[slot].n_loads);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_empty[slot]));
                 if (g >= total_items) break;
-                if (t >= item.n_sides) {
-                    ring_base += (uint32_t)item.n_loads;
-                    kv_walk(ring_base);
-                    continue;
-                }
-                const clear_pair_step_t *steps = prm.steps + item.step_begin;
-                const int n = item.step_count;
-                ok = wait_bar(ptx::smem_u32(&ctrl->q_full[t]), n_it & 1u, abort_flag, prm.status, 6);
+                const clear_pair_step_t *steps = prm.steps + step_begin;
+                for (int t = 0; t < n_sides && ok; ++t)
+                    ok = __all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->q_full[t]), n_it[t] & 1u, abort_flag, prm.status, 6));
                 if (!ok) break;
 
-                // S_t = Q_t K^T for the key tile of `st`; both operands K-major: 16 contraction channels
-                // are 32 bytes along a 128-byte row, the next 64 channels are the tile's second half.
-                auto issue_qk = [&](const clear_pair_step_t &st) {
-                    // the softmax warps must have taken the previous S_t out of tensor memory
-                    if (n_qk > 0) ok = wait_bar(b_sfree, (n_qk - 1) & 1u, abort_flag, prm.status, 16);
+                // One group of MMAs for query tile t: O_t += P_t V of its previous step (if one is pending:
+                // pv), then S_t = Q_t K^T of this step (if it takes part: qk).  Everything that does not
+                // need P_t -- the fills of the V and K stages, the descriptors -- comes before the wait for
+                // P_t, so that between the arrival of P_t and the MMAs lie as few instructions as possible:
+                // this warp shares its scheduler with two softmax warps in their exponential phase.
+                //   P_t V : P_t (bf16 pairs) in the first 64 columns of S_t, 16 keys = 8 columns; V MN-major,
+                //           16 keys are 16 rows of 128 bytes = 2048 bytes;
+                //   Q K^T : both operands K-major: 16 contraction channels are 32 bytes along a 128-byte row,
+                //           the next 64 channels are the tile's second half.
+                auto issue_group = [&](int t, bool pv, int pv_flags, int pv_base, bool first_pv, bool qk, int qk_flags,
+                                       int qk_base, bool last) {
+                    const bool pv_shared = (pv_flags & CLEAR_STEP_SHARED) != 0, qk_shared = (qk_flags & CLEAR_STEP_SHARED) != 0;
+                    const uint32_t pos_v = ring_base + ((uint32_t)pv_base >> 16) + (uint32_t)step_tile_index(pv_flags, t);
+                    const uint32_t pos_k = ring_base + ((uint32_t)qk_base & 0xffffu) + (uint32_t)step_tile_index(qk_flags, t);
+                    TRACE_MARK(0)
+                    if (pv && !(pv_shared && t == 1)) kv_wait(pos_v);
+                    if (qk && !(qk_shared && t == 1)) kv_wait(pos_k);
+                    // the epilogue must have read the previous item's O_t out of tensor memory
+                    if (ok && pv && first_pv)
+                        ok = __all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->o_empty[t]), (n_it[t] & 1u) ^ 1u, abort_flag, prm.status, 8));
+                    TRACE_MARK(1)  // wait for K, V
+                    const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
+                    const uint32_t v_lo = ptx::smem_desc_lo(sRing + (pos_v % kRing) * kTileBytes, kHalfBytes);
+                    const uint32_t q_lo = ptx::smem_desc_lo(sQ + t * kTileBytes, 16);
+                    const uint32_t k_lo = ptx::smem_desc_lo(sRing + (pos_k % kRing) * kTileBytes, 16);
+                    const uint32_t b_vfree = ptx::smem_u32(&ctrl->kv_empty[pos_v % kRing]);
+                    const uint32_t b_kfree = ptx::smem_u32(&ctrl->kv_empty[pos_k % kRing]);
+                    const bool free_v = !pv_shared || t == 1, free_k = !qk_shared || t == 1;
+                    if (ok && pv) ok = __all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->p_ready[t]), n_pv[t] & 1u, abort_flag, prm.status, 7));
                     if (!ok) return;
-                    const uint32_t pos = ring_base + ((uint32_t)st.load_base & 0xffffu) + (uint32_t)step_tile_index(st.flags, t);
-                    const uint32_t stage = kv_wait(pos);
-                    if (!ok) return;
+                    TRACE_MARK(4)  // wait for P
                     ptx::tc_fence_after();
-                    const uint32_t k_lo = ptx::smem_desc_lo(sRing + stage * kTileBytes, 16);
-                    ptx::mma_ss_c<false>(tmem_S, ptx::make_desc(q_lo, kDescHiK), ptx::make_desc(k_lo, kDescHiK), kIdescQK);
+                    if (ptx::elect_one()) {
+                        if (pv) {
+                            ptx::mma_ts(tmem_O, tmem_S, ptx::make_desc(v_lo, kDescHiK), kIdescPV, first_pv ? 0u : 1u);
 #pragma unroll
-                    for (int kk = 1; kk < D / 16; ++kk) {
-                        const uint32_t off16 = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
-                        ptx::mma_ss_c<true>(tmem_S, ptx::make_desc(q_lo + off16, kDescHiK),
-                                            ptx::make_desc(k_lo + off16, kDescHiK), kIdescQK);
-                    }
-                    ptx::tc_commit(b_sfull);
-                    kv_release(stage);
-                    ++n_qk;
-                };
-                auto v_position = [&](const clear_pair_step_t &st) -> uint32_t {
-                    return ring_base + ((uint32_t)st.load_base >> 16) + (uint32_t)step_tile_index(st.flags, t);
-                };
-
-                // first step this query tile takes part in (every tile has at least one)
-                int s = 0;
-                clear_pair_step_t cur = load_step(steps);
-                while (!step_uses(cur.flags, t) && s + 1 < n) cur = load_step(steps + ++s);
-                clear_pair_step_t pre = cur;  // record s + 1, fetched one step ahead
-                if (s + 1 < n) pre = load_step(steps + s + 1);
-                issue_qk(cur);
-                bool first_pv = true;
-                while (ok) {
-                    // next step of this query tile
-                    int s2 = s + 1;
-                    clear_pair_step_t nxt = pre;
-                    while (s2 < n && !step_uses(nxt.flags, t)) {
-                        ++s2;
-                        if (s2 < n) nxt = load_step(steps + s2);
-                    }
-                    const bool has_next = s2 < n;
-                    if (has_next && s2 + 1 < n) pre = load_step(steps + s2 + 1);
-                    // every Q_t K^T of the item has been issued: the next item's Q tile may land
-                    if (!has_next) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
-
-                    const uint32_t pos_v = v_position(cur);
-                    // The next S_t goes ahead of this step's P_t V whenever its K tile was staged before this
-                    // step's V tile (it is, unless this query tile sits out the steps in between): the ring
-                    // is walked in staging order.
-                    bool qk_done = false;
-                    if (has_next) {
-                        const uint32_t pos_k = ring_base + ((uint32_t)nxt.load_base & 0xffffu) + (uint32_t)step_tile_index(nxt.flags, t);
-                        if (pos_k < pos_v) {
-                            issue_qk(nxt);
-                            qk_done = true;
-                            if (!ok) break;
+                            for (int kk = 1; kk < 8; ++kk)
+                                ptx::mma_ts_c<true>(tmem_O, tmem_S + kk * 8, ptx::make_desc(v_lo + kk * (2048 >> 4), kDescHiK), kIdescPV);
+                            if (free_v) ptx::tc_commit(b_vfree);
                         }
-                    }
-
-                    // O_t += P_t V, the two 64-key halves of P one after the other
-                    if (!qk_done) kv_walk(pos_v);
-                    uint32_t stage_v = 0;
+                        if (qk) {
+                            ptx::mma_ss_c<false>(tmem_S, ptx::make_desc(q_lo, kDescHiK), ptx::make_desc(k_lo, kDescHiK), kIdescQK);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (h == 0) {
-                            ok = wait_bar(ptx::smem_u32(&ctrl->p_ready[t]), n_pv & 1u, abort_flag, prm.status, 7);
-                            if (!ok) break;
-                            stage_v = kv_wait(pos_v);
-                            if (!ok) break;
-                            if (first_pv) {
-                                // the epilogue must have read the previous item's O_t out of tensor memory
-                                ok = wait_bar(ptx::smem_u32(&ctrl->o_empty[t]), (n_it & 1u) ^ 1u, abort_flag, prm.status, 8);
-                                if (!ok) break;
+                            for (int kk = 1; kk < D / 16; ++kk) {
+                                const uint32_t off16 = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                                ptx::mma_ss_c<true>(tmem_S, ptx::make_desc(q_lo + off16, kDescHiK),
+                                                    ptx::make_desc(k_lo + off16, kDescHiK), kIdescQK);
                             }
+                            ptx::tc_commit(ptx::smem_u32(&ctrl->s_full[t]));
+                            if (free_k) ptx::tc_commit(b_kfree);
                         }
-                        ptx::tc_fence_after();
-                        // P half: K-major, 16 keys are 32 bytes along a row; V: MN-major, 16 keys are 16
-                        // rows of 128 bytes = 2048 bytes
-                        const uint32_t v_lo = ptx::smem_desc_lo(sRing + stage_v * kTileBytes, kHalfBytes) + h * 4 * (2048 >> 4);
-                        const uint32_t ph_lo = p_lo + h * (kHalfBytes >> 4);
-                        ptx::mma_ss(tmem_O, ptx::make_desc(ph_lo, kDescHiK), ptx::make_desc(v_lo, kDescHiK), kIdescPV,
-                                    (first_pv && h == 0) ? 0u : 1u);
+                        // the item's last group of the tile: its output is complete once these MMAs are
+                        if (last) ptx::tc_commit(ptx::smem_u32(&ctrl->o_full[t]));
+                    }
+                    __syncwarp();
+                    if (pv) ++n_pv[t];
+                    TRACE_MARK(5)  // issue
+                };
+
+                int pend_flags[2] = {0, 0}, pend_base[2] = {0, 0};  // the step whose P_t V is still to be issued
+                bool pending[2] = {false, false};
+                bool first_pv[2] = {true, true};
+                int4 rec = __ldg(reinterpret_cast<const int4 *>(steps) + 1);  // flags, n_valid0, n_valid1, load_base
+                for (int s = 0; s < n && ok; ++s) {
+                    const int flags = uni(rec.x), load_base = uni(rec.w);
+                    if (s + 1 < n) rec = __ldg(reinterpret_cast<const int4 *>(steps + s + 1) + 1);  // one step ahead
 #pragma unroll
-                        for (int kk = 1; kk < 4; ++kk)
-                            ptx::mma_ss_c<true>(tmem_O, ptx::make_desc(ph_lo + kk * 2, kDescHiK),
-                                                ptx::make_desc(v_lo + kk * (2048 >> 4), kDescHiK), kIdescPV);
-                        // P may be overwritten (and O_t rescaled) once this step's MMAs have retired
-                        if (h == 1) ptx::tc_commit(b_pfree);
+                    for (int t = 0; t < 2; ++t) {
+                        if (t >= n_sides || !ok) continue;
+                        const bool qk = step_uses(flags, t);
+                        if (!pending[t] && !qk) continue;
+                        issue_group(t, pending[t], pend_flags[t], pend_base[t], first_pv[t], qk, flags, load_base, false);
+                        if (pending[t]) first_pv[t] = false;
+                        pending[t] = qk;
+                        pend_flags[t] = flags;
+                        pend_base[t] = load_base;
                     }
-                    if (!ok) break;
-                    first_pv = false;
-                    ++n_pv;
-                    kv_release(stage_v);
-                    if (!has_next) {
-                        ptx::tc_commit(ptx::smem_u32(&ctrl->o_full[t]));
-                        break;
-                    }
-                    if (!qk_done) issue_qk(nxt);
-                    cur = nxt;
-                    s = s2;
                 }
-                ++n_it;
-                ring_base += (uint32_t)item.n_loads;
-                kv_walk(ring_base);
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t >= n_sides || !ok) continue;
+                    // every Q_t K^T of the item has been issued: the next item's Q tile may land
+                    if (ptx::elect_one()) ptx::tc_commit(ptx::smem_u32(&ctrl->q_empty[t]));
+                    __syncwarp();
+                    issue_group(t, pending[t], pend_flags[t], pend_base[t], first_pv[t], false, 0, 0, true);
+                    ++n_it[t];
+                }
+                ring_base += (uint32_t)n_loads;
             }
+#ifdef CLEAR_WS_TRACE
+            TRACE_MARK(0)
+            if (blockIdx.x == 0 && lane == 0)
+                printf("mma thread: other %llu waitK %llu issueQK %llu waitV %llu waitP %llu issuePV %llu\n", tr_acc[0], tr_acc[1],
+                       tr_acc[2], tr_acc[3], tr_acc[4], tr_acc[5]);
+#endif
             if (*abort_flag) {
                 // MMAs that were issued must retire before tensor memory is given back
-                ptx::tc_commit(ptx::smem_u32(&ctrl->drain[t]));
-                drain_bar(ptx::smem_u32(&ctrl->drain[t]), 0);
+                if (lane == 0) {
+                    ptx::tc_commit(ptx::smem_u32(&ctrl->drain[0]));
+                    drain_bar(ptx::smem_u32(&ctrl->drain[0]), 0);
+                }
             }
         }
         __syncwarp();
     } else {
         // ================= softmax warps: thread r owns query row r (tensor-memory lane r) of its tile =====
-        // Per step: S_t into registers (the next Q_t K^T may then overwrite it), Eq. 3 mask, row maximum,
-        // P = exp2(.) as bf16 into shared memory with the row sum; at the end of an item O_t / l -> bf16 ->
-        // global memory (or fp32 partial results of split text rows).
+        // Per step: S_t into registers, row maximum, P = exp2(.) under the Eq. 3 mask as bf16 into tensor
+        // memory over S_t, row sum; at the end of an item O_t / l -> bf16 -> global memory (or fp32 partial
+        // results of split text rows).
         ptx::setmaxnreg_inc<kRegsSoftmax>();
+        TRACE_DECL
         const int t = (warp - 4) >> 2;  // query tile of the pair
         const int q4 = warp & 3;        // tensor-memory lane quadrant
         const int r = q4 * 32 + lane;   // query row of the tile
         const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
         const uint32_t tmem_S = tmem + t * 128, tmem_O = tmem + 256 + t * 128;
         const float c = prm.scale_log2;
-        const uint32_t b_s = ptx::smem_u32(&ctrl->s_full[t]), b_sfree = ptx::smem_u32(&ctrl->s_free[t]);
-        const uint32_t b_pfree = ptx::smem_u32(&ctrl->p_free[t]), b_pready = ptx::smem_u32(&ctrl->p_ready[t]);
-        // this row of the two P half-tiles (64 keys each): K-major, 128-byte rows, 16-byte chunks
-        // XOR-swizzled by the row number
-        const uint32_t p_row = sP + t * 2 * kHalfBytes + r * 128;
-        uint32_t p_chunk[8];  // where the eight 16-byte chunks of a row go
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) p_chunk[ch] = p_row + (uint32_t)((ch ^ (r & 7)) << 4);
+        const uint32_t b_s = ptx::smem_u32(&ctrl->s_full[t]), b_pready = ptx::smem_u32(&ctrl->p_ready[t]);
         uint32_t n_s = 0, n_items_seen = 0;
         bool alive = true;
         for (uint32_t k = 0; alive; ++k) {
@@ -575,7 +543,6 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             const bool q_valid = is_text ? r < (t ? item.n_rows1 : item.n_rows0) : (q_y < prm.grid_h && q_x < prm.grid_w);
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
-            bool prev_shared = false;
 
             // Step records are fetched two steps ahead and this row's precomputed mask words one step ahead,
             // so that neither latency is on the critical path.
@@ -589,15 +556,14 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
             SideStep st_next2 = st_next;
             if (step_count > 1) st_next2 = load_side_step(steps + 1, t);
             uint4 mrow_next = load_mask_row(st_next);
+            TRACE_MARK(8)  // between items
             for (int s = 0; s < step_count; ++s) {
                 const SideStep st = st_next;
                 const uint4 mrow = mrow_next;
                 st_next = st_next2;  // fetched a step ago: the mask row's address does not wait for it
                 if (s + 2 < step_count) st_next2 = load_side_step(steps + s + 2, t);
-                if (!step_uses(st.flags, t)) {
-                    if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
-                    continue;
-                }
+                if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
+                if (!step_uses(st.flags, t)) continue;
                 const bool masked = (st.flags & kMaskedBit) != 0;
                 // ---- mask bits of this row for the tile (bit j of word w = key 32 w + j allowed) --------
                 uint32_t mw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
@@ -651,129 +617,135 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     }
                 }
 
-                // warp-uniform outcome: the tcgen05.ld / st below need the whole warp
+                TRACE_MARK(0)  // step prologue: records, mask words
+                // warp-uniform outcome: the tcgen05.ld / st below need the whole warp.  Once S_t of this step
+                // is complete, so is P_t V of the step before (same thread, same pipe, issued earlier).
                 if (!__all_sync(0xffffffffu, wait_bar(b_s, n_s & 1u, abort_flag, prm.status, 10))) {
                     alive = false;
                     break;
                 }
                 ++n_s;
+                TRACE_MARK(1)  // wait for S
                 ptx::tc_fence_after();
                 uint32_t sv[4][32];
 #pragma unroll
                 for (int w = 0; w < 4; ++w) ptx::tmem_ld32(tmem_S + lane_off + 32 * w, sv[w]);
                 ptx::tmem_wait_ld();
-                // S_t is in registers: the next Q_t K^T may overwrite it
-                ptx::tc_fence_before();
-                warp_arrive(b_sfree, lane);
-                if (s + 1 < step_count) mrow_next = load_mask_row(st_next);
+                TRACE_MARK(2)  // S into registers
 
-                // row maximum over the allowed keys, four independent chains of three-input maxima
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                if (masked) {
+                // ---- P = exp2(S * c - m * c) on the allowed keys, 0 elsewhere; row sum; bf16 pairs into
+                // tensor memory, 32 keys (16 columns) at a time (two-wide fp32 FMA and ADD; four independent
+                // partial sums)
+                float tile_sum = 0.f;
+                auto exp_pass = [&](auto masked_c, float mc) {
+                    constexpr bool kMasked = decltype(masked_c)::value;
+                    const uint64_t c2 = ptx::pack2(c, c), nmc2 = ptx::pack2(-mc, -mc);
+                    uint64_t lsum[2] = {0ull, 0ull};
 #pragma unroll
-                    for (int w = 0; w < 4; ++w)
+                    for (int w = 0; w < 4; ++w) {
+                        uint32_t pk[16];
 #pragma unroll
                         for (int j = 0; j < 32; j += 2) {
-                            const float v0 = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
-                            const float v1 = ((mw[w] >> (j + 1)) & 1u) ? __uint_as_float(sv[w][j + 1]) : -INFINITY;
-                            sv[w][j] = __float_as_uint(v0);
-                            sv[w][j + 1] = __float_as_uint(v1);
-                            mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], v0, v1);
-                        }
-                } else {
-#pragma unroll
-                    for (int w = 0; w < 4; ++w)
-#pragma unroll
-                        for (int j = 0; j < 32; j += 2)
-                            mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], __uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1]));
-                }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-
-                // The previous step's P_t V must have retired before O_t is rescaled or P is written again
-                // (the barrier completes once per step).
-                if (n_s > 1) {
-                    if (!__all_sync(0xffffffffu, wait_bar(b_pfree, n_s & 1u, abort_flag, prm.status, 17))) {
-                        alive = false;
-                        break;
-                    }
-                    ptx::tc_fence_after();
-                }
-                // ---- running maximum; O is rescaled only when it grew by more than the threshold -----
-                const float m_new = fmaxf(m_used, mx);
-                if (first) {
-                    m_used = m_new;
-                    first = false;
-                } else {
-                    const bool need = (m_new - m_used) * c > kRescaleThreshold;  // false for NaN (-inf minus -inf)
-                    if (__any_sync(0xffffffffu, need)) {
-                        float alpha = 1.f;
-                        if (need) {
-                            alpha = ptx::ex2((m_used - m_new) * c);
-                            m_used = m_new;
-                            l *= alpha;
-                        }
-#pragma unroll 1
-                        for (int w = 0; w < D / 16; ++w) {
-                            uint32_t o[16];
-                            ptx::tmem_ld16(tmem_O + lane_off + 16 * w, o);
-                            ptx::tmem_wait_ld();
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-                            ptx::tmem_st16(tmem_O + lane_off + 16 * w, o);
-                        }
-                        ptx::tmem_wait_st();
-                        ptx::tc_fence_before();
-                    }
-                }
-                {
-                    const bool shared = (st.flags & CLEAR_STEP_SHARED) != 0;
-                    if (t == 1 && shared && !prev_shared) {
-                        const long long t0 = clock64();
-                        while (clock64() - t0 < kStaggerClocks) {
-                        }
-                    }
-                    prev_shared = shared;
-                }
-                const float mc = (m_used == -INFINITY) ? 0.f : m_used * c;
-
-                // ---- P = exp2(S * c - m * c), row sum, bf16 pairs into the P half-tiles -----------------
-                // (two-wide fp32 FMA and ADD; four independent partial sums)
-                const uint64_t c2 = ptx::pack2(c, c), nmc2 = ptx::pack2(-mc, -mc);
-                uint64_t lsum[2] = {0ull, 0ull};
-#pragma unroll
-                for (int w = 0; w < 4; ++w) {
-#pragma unroll
-                    for (int grp = 0; grp < 2; ++grp) {
-                        uint32_t pk[8];  // 16 keys = two 16-byte chunks of the row
-#pragma unroll
-                        for (int j = 16 * grp; j < 16 * grp + 16; j += 2) {
                             const uint64_t x2 =
                                 ptx::fma2(ptx::pack2(__uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1])), c2, nmc2);
                             float x0, x1;
                             ptx::unpack2(x2, x0, x1);
+                            if (kMasked) {
+                                x0 = ((mw[w] >> j) & 1u) ? x0 : -INFINITY;
+                                x1 = ((mw[w] >> (j + 1)) & 1u) ? x1 : -INFINITY;
+                            }
                             const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);
                             lsum[(j >> 1) & 1] = ptx::add2(lsum[(j >> 1) & 1], ptx::pack2(p0, p1));
-                            pk[(j >> 1) & 7] = ptx::pack_bf16(p0, p1);
+                            pk[j >> 1] = ptx::pack_bf16(p0, p1);
                         }
-#pragma unroll
-                        for (int cc = 0; cc < 2; ++cc) {
-                            const int ch = 4 * (w & 1) + 2 * grp + cc;  // chunk of the 128-byte row of half w / 2
-                            ptx::st_shared_v4(p_chunk[ch] + (w >> 1) * kHalfBytes, pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2],
-                                              pk[4 * cc + 3]);
-                        }
+                        ptx::tmem_st16(tmem_S + lane_off + 16 * w, pk);
                     }
-                }
-                // generic-proxy writes -> visible to the tensor core's (async proxy) reads
-                ptx::fence_proxy_async_smem();
-                warp_arrive(b_pready, lane);
-                {
                     float a0, a1, a2, a3;
                     ptx::unpack2(lsum[0], a0, a1);
                     ptx::unpack2(lsum[1], a2, a3);
-                    l += (a0 + a1) + (a2 + a3);
+                    tile_sum = (a0 + a1) + (a2 + a3);
+                };
+                // The running maximum m of a row moves only when a tile's maximum over the allowed keys
+                // exceeds it by more than the threshold, i.e. when some P of the tile would exceed
+                // 2^threshold.  So P is formed against the maximum as it stands, and only when a row's sum
+                // over the tile exceeds 2^threshold (no single P can otherwise), or the row has no maximum
+                // yet, is the tile's maximum taken, m moved by the rule above, O rescaled and P formed again:
+                // the same results as with a maximum pass on every tile, which costs a third of the
+                // exponentials' time and is needed on the first tile of a row and hardly ever after.
+                bool use_mask = masked;
+                bool exact = __any_sync(0xffffffffu, first || (m_used == -INFINITY && q_valid));
+#pragma unroll 1
+                for (;;) {
+                    if (exact) {
+                        // maximum over the allowed keys (the scores Eq. 3 forbids become -inf in place)
+                        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                        if (use_mask) {
+#pragma unroll
+                            for (int w = 0; w < 4; ++w)
+#pragma unroll
+                                for (int j = 0; j < 32; j += 2) {
+                                    const float v0 = ((mw[w] >> j) & 1u) ? __uint_as_float(sv[w][j]) : -INFINITY;
+                                    const float v1 = ((mw[w] >> (j + 1)) & 1u) ? __uint_as_float(sv[w][j + 1]) : -INFINITY;
+                                    sv[w][j] = __float_as_uint(v0);
+                                    sv[w][j + 1] = __float_as_uint(v1);
+                                    mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], v0, v1);
+                                }
+                            use_mask = false;
+                        } else {
+#pragma unroll
+                            for (int w = 0; w < 4; ++w)
+#pragma unroll
+                                for (int j = 0; j < 32; j += 2)
+                                    mx4[(j >> 1) & 3] = ptx::max3(mx4[(j >> 1) & 3], __uint_as_float(sv[w][j]), __uint_as_float(sv[w][j + 1]));
+                        }
+                        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                        const float m_new = fmaxf(m_used, mx);
+                        if (first) {
+                            m_used = m_new;
+                        } else {
+                            const bool need = (m_new - m_used) * c > kRescaleThreshold;  // false for NaN (-inf minus -inf)
+                            if (__any_sync(0xffffffffu, need)) {
+                                float alpha = 1.f;
+                                if (need) {
+                                    alpha = ptx::ex2((m_used - m_new) * c);
+                                    m_used = m_new;
+                                    l *= alpha;
+                                }
+#pragma unroll 1
+                                for (int w = 0; w < D / 16; ++w) {
+                                    uint32_t o[16];
+                                    ptx::tmem_ld16(tmem_O + lane_off + 16 * w, o);
+                                    ptx::tmem_wait_ld();
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                                    ptx::tmem_st16(tmem_O + lane_off + 16 * w, o);
+                                }
+                            }
+                        }
+                    }
+                    const float mc = (m_used == -INFINITY) ? 0.f : m_used * c;
+                    if (use_mask)
+                        exp_pass(std::true_type{}, mc);
+                    else
+                        exp_pass(std::false_type{}, mc);
+                    if (exact) break;
+                    exact = __any_sync(0xffffffffu, !(tile_sum <= kMaxTileSum));  // also for a NaN
+                    if (!exact) break;
                 }
+                first = false;
+                l += tile_sum;
+                TRACE_MARK(5)  // exponentials
+                // P_t (and a rescaled O_t) must be in tensor memory before the MMA thread is told
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before();
+                warp_arrive(b_pready, lane);
+                TRACE_MARK(6)  // arrival
+#ifdef CLEAR_WS_TRACE
+                ++tr_steps;
+#endif
             }
             if (!alive) break;
+            TRACE_MARK(0)
 
             // ---- epilogue: the last P_t V has retired once o_full completes; O_t / l -> global memory -----
             if (!__all_sync(0xffffffffu, wait_bar(ptx::smem_u32(&ctrl->o_full[t]), n_items_seen & 1u, abort_flag, prm.status, 14)))
@@ -830,7 +802,13 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     }
                 }
             }
+            TRACE_MARK(7)  // epilogue
         }
+#ifdef CLEAR_WS_TRACE
+        if (blockIdx.x == 0 && lane == 0)
+            printf("tile %d warp %d steps %u: prologue %llu waitS %llu ldS %llu max %llu rescale %llu exp %llu arrive %llu epilogue %llu between items %llu\n",
+                   t, q4, tr_steps, tr_acc[0], tr_acc[1], tr_acc[2], tr_acc[3], tr_acc[4], tr_acc[5], tr_acc[6], tr_acc[7], tr_acc[8]);
+#endif
     }
 
     ptx::tc_fence_before();
@@ -922,7 +900,7 @@ std::mutex g_dev_mutex;
 template <int D>
 int launch_variant(const clear_plan &p, const CUtensorMap *tm, const WsParams &prm, cudaStream_t stream)
 {
-    constexpr size_t kSmem = (size_t)(2 + kRing) * (D / 64) * 16384 + 4 * 16384 + sizeof(Ctrl);
+    constexpr size_t kSmem = (size_t)(2 + kRing) * (D / 64) * 16384 + sizeof(Ctrl);
     static_assert(kSmem <= 232448, "shared memory of one block");
     int n_sm = 0;
     {

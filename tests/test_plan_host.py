@@ -251,14 +251,13 @@ def test_pair_schedule_covers_each_allowed_pair_exactly_once(gh, gw, T, r):
         assert it.step_count >= 1 and it.n_sides in (1, 2)
         sts = steps[it.step_begin: it.step_begin + it.step_count]
         # ring bookkeeping: K and V of each distinct key tile of a step take one stage each, in the order
-        # K(0), then K(s + 1), V(s) for every step s
+        # K(s), V(s) for every step s
         def tiles_of(st):
             return int(bool(st.flags & clear.STEP_USE0)) + int(bool(st.flags & clear.STEP_USE1) and
                                                                not st.flags & clear.STEP_SHARED)
-        order = [("K", 0)]
+        order = []
         for i in range(len(sts)):
-            if i + 1 < len(sts):
-                order.append(("K", i + 1))
+            order.append(("K", i))
             order.append(("V", i))
         pos, where = 0, {}
         for kind, i in order:
@@ -385,3 +384,17 @@ def test_text_rows_are_split_for_long_sequences():
     assert len(interior) > 1500                          # 15 key patches + 4 text tiles away from borders
     g = info.sum_mask / info.executed_pairs
     assert 0.55 < g < 0.70
+
+
+def test_key_lists_beyond_the_step_records_positions_fall_back():
+    """A pair item that stages more than 65535 key / value tiles cannot be named by the 16-bit ring positions of
+    the step records: the warp-specialised kernel refuses the shape, and a plan that leaves the choice to the
+    library runs it on the CUDA-core kernel."""
+    gh = gw = 2048          # 32768 key patches, every one within reach of every query patch at this radius
+    with pytest.raises(clear.ClearError) as e:
+        clear.Plan(1, 1, gh, gw, 0, 128, 4096.0, kernel=clear.KERNEL_TCGEN05_WS, host_only=True)
+    assert e.value.status == clear.ERR_UNSUPPORTED
+    p = clear.Plan(1, 1, gh, gw, 0, 128, 4096.0, host_only=True)
+    assert p.info().kernel == clear.KERNEL_SIMT
+    n = gh * gw
+    assert p.info().sum_mask == n * n
