@@ -145,7 +145,14 @@ typedef struct clear_pair_item {
 
 /* Eq. 1 under the mask of Eq. 3 for bf16 tensors, fp32 accumulation, bf16 output.
  * A plan for the shape is looked up in (or added to) a process-wide cache, so the first call for
- * a shape allocates and copies small tables; later calls only launch kernels.
+ * a shape allocates and copies small tables; later calls only launch kernels.  The cache keeps the
+ * 16 most recently used plans (environment variable CLEAR_CACHE_MAX_PLANS); making room for a new
+ * shape synchronises the device.
+ * Streams and threads: any.  Calls for one shape share one plan (work queue, status words, split-KV
+ * workspace), so the library orders them on the device: a call made on another stream than the call
+ * before it for that shape first waits there for that call's kernels (cudaStreamWaitEvent, no host
+ * wait).  Calls for different shapes, or on different devices, do not wait for each other.
+ * A kernel whose bounded wait expired is found by clear_cache_check, not here.
  * Errors: INVALID_ARG (B, H, grid_h, grid_w, head_dim <= 0; n_text < 0; radius <= 0 or
  * non-finite; scale non-finite; null tensor), MISALIGNED, UNSUPPORTED (head_dim > 256), CUDA. */
 int clear_attn_fwd(const void *q, const void *k, const void *v, void *out, int B, int H, int grid_h,
@@ -192,7 +199,8 @@ int clear_plan_pair_tables(const clear_plan_t *plan, const clear_pair_item_t **i
 int clear_plan_mask_table(const clear_plan_t *plan, const uint32_t **words, int32_t *n_entries);
 
 /* Forward pass with an explicit plan.  Tensor dtype is the plan's.  Calls on one plan share its
- * workspace: run them on one stream, or order them yourself.
+ * workspace and work queue; the library orders them on the device as described at clear_attn_fwd, so
+ * they may be made on any streams (two plans of one shape run side by side).
  * Errors: INVALID_ARG, MISALIGNED, PLAN_MISMATCH (current device differs from the plan's),
  * UNSUPPORTED (tensor-core plan called with scale <= 0), CUDA. */
 int clear_attn_fwd_planned(const clear_plan_t *plan, const void *q, const void *k, const void *v,
@@ -227,9 +235,12 @@ int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_ho
  * and a split-KV workspace per plan; this one keeps them in one file-scope device array inside the
  * library image, so every GPU that loads the library holds those ~33.3 MiB until the process exits.
  *
- * Same tensors, layout and mathematics as clear_attn_fwd (results are identical bit for bit); head_dim
- * must be 64 or 128 and scale > 0.  It calls no cudaMalloc / cudaFree and no allocating library routine;
- * it does enqueue small table copies and one 4-byte memset on `stream`.
+ * Same tensors, layout and mathematics as clear_attn_fwd; it runs the one-tile-per-block tensor-core
+ * kernel, so its results equal those of a CLEAR_KERNEL_TCGEN05 plan bit for bit and those of
+ * clear_attn_fwd (another kernel) within the bf16 tolerance.  head_dim must be 64 or 128 and scale > 0.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine; it does enqueue one 4-byte memset
+ * on `stream` and, when the shape differs from the previous call's, three small table copies from
+ * ordinary host memory (such a copy can make the host wait for the stream).
  * - The first call on a device looks up the array's device address (set-up); make that call with the
  *   device current and before starting any stream capture.
  * - Shapes whose tables or partial results exceed the CLEAR_STATIC_* capacities are rejected with
@@ -245,15 +256,28 @@ int clear_attn_fwd_static(const void *q, const void *k, const void *v, void *out
 /* Fill `info` from the plan (host only, no CUDA call).  Errors: INVALID_ARG. */
 int clear_plan_info(const clear_plan_t *plan, clear_plan_info_t *info);
 
-/* Synchronise `stream`, then read and clear the plan's device status word.  Returns
+/* Synchronise `stream`, then read and clear the plan's device status words.  Returns
  * CLEAR_ERR_DEVICE_TIMEOUT if any kernel launched with this plan gave up on a bounded wait since
- * the last check, CLEAR_OK otherwise.  Errors: INVALID_ARG, CUDA. */
+ * the last check, CLEAR_OK otherwise.  A launch whose blocks gave up writes nothing more (its outputs
+ * are incomplete); later launches of the plan run normally.  Errors: INVALID_ARG, CUDA. */
 int clear_plan_check(clear_plan_t *plan, void *stream);
+
+/* Give back the staging buffers (four tensors' worth of device memory) and the copy pipeline that
+ * clear_attn_fwd_host built for this plan; the next such call builds them again.  Synchronises the
+ * plan's device.  Errors: INVALID_ARG, CUDA. */
+int clear_plan_trim(clear_plan_t *plan);
 
 /* Free the plan's device memory and the handle.  NULL is accepted.  Errors: CUDA. */
 int clear_plan_destroy(clear_plan_t *plan);
 
-/* Drop every plan the unplanned entry points cached (synchronises the device first). */
+/* clear_plan_check for every plan the unplanned entry points (clear_attn_fwd, clear_attn_fwd_f32)
+ * have cached for the current device: waits for their last launches and for `stream`, returns
+ * CLEAR_ERR_DEVICE_TIMEOUT if a kernel of any of them gave up on a bounded wait since the last check
+ * (clear_last_device_status names the wait), and clears that record.  Errors: CUDA. */
+int clear_cache_check(void *stream);
+
+/* Drop every plan the unplanned entry points cached (synchronises the device first; no call of those
+ * entry points runs at the same time: they hold the cache's lock while they launch). */
 int clear_cache_clear(void);
 
 /* Static, human-readable name of a status code. */

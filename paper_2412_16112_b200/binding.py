@@ -27,7 +27,7 @@ EXPORTS = [
     "clear_plan_tables", "clear_attn_fwd_planned", "clear_attn_fwd_host", "clear_plan_info",
     "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
     "clear_last_cuda_error", "clear_attn_fwd_static", "clear_plan_pair_tables",
-    "clear_last_device_status", "clear_plan_mask_table",
+    "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim",
 ]
 
 
@@ -109,6 +109,8 @@ def load() -> ctypes.CDLL:
         lib.clear_plan_check.argtypes = [vp, vp]
         lib.clear_plan_destroy.argtypes = [vp]
         lib.clear_cache_clear.argtypes = []
+        lib.clear_cache_check.argtypes = [vp]
+        lib.clear_plan_trim.argtypes = [vp]
         lib.clear_status_string.argtypes = [i32]
         lib.clear_status_string.restype = ctypes.c_char_p
         lib.clear_last_cuda_error.argtypes = []
@@ -255,6 +257,9 @@ class Plan:
     def check(self, stream=None) -> None:
         _check(load().clear_plan_check(self._h, _stream_ptr(stream)), "clear_plan_check")
 
+    def trim(self) -> None:
+        _check(load().clear_plan_trim(self._h), "clear_plan_trim")
+
     def destroy(self) -> None:
         if self._h:
             load().clear_plan_destroy(self._h)
@@ -269,3 +274,7 @@ class Plan:
 
 def clear_cache_clear() -> None:
     _check(load().clear_cache_clear(), "clear_cache_clear")
+
+
+def clear_cache_check(stream=None) -> None:
+    _check(load().clear_cache_check(_stream_ptr(stream)), "clear_cache_check")

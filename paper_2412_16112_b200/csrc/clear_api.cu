@@ -51,6 +51,10 @@ int free_device_parts(clear_plan *p)
     rel(p->d_status);
     rel(p->d_partial_o);
     rel(p->d_partial_ml);
+    if (p->ev_last) {
+        (void)cudaEventDestroy(p->ev_last);
+        p->ev_last = nullptr;
+    }
     for (void *&s : p->d_stage) {
         rel(s);
         s = nullptr;
@@ -120,6 +124,14 @@ int create_plan(clear_plan_t **out, const Shape &shape_in, bool host_only)
         if (rc == CLEAR_OK) {
             cudaError_t e = cudaMalloc((void **)&p->d_status, kStatusWords * sizeof(int));
             if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, kStatusWords * sizeof(int));
+            // For tests of the error path: the status word starts as if a bounded wait of an earlier block
+            // had expired, so the plan's first launch takes the early-leave path (no wait is made to expire).
+            if (e == cudaSuccess)
+                if (const char *preset = std::getenv("CLEAR_TEST_PRESET_STATUS")) {
+                    const int code = std::atoi(preset);
+                    if (code != 0) e = cudaMemcpy(p->d_status, &code, sizeof(int), cudaMemcpyHostToDevice);
+                }
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_last, cudaEventDisableTiming);
             if (e != cudaSuccess) {
                 note_cuda_error((int)e);
                 (void)cudaGetLastError();
@@ -241,9 +253,20 @@ int forward(const clear_plan *p, const void *q, const void *k, const void *v, vo
     CLEAR_CUDA_TRY(cudaGetDevice(&dev));
     if (dev != p->device) return CLEAR_ERR_PLAN_MISMATCH;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (p->kernel == CLEAR_KERNEL_TCGEN05) return launch_tc(*p, q, k, v, out, scale, st);
-    if (p->kernel == CLEAR_KERNEL_TCGEN05_WS) return launch_ws(*p, q, k, v, out, scale, st);
-    return launch_simt(*p, q, k, v, out, scale, st);
+    // launches of one plan run one after the other on the device, whatever streams they are made on
+    std::lock_guard<std::mutex> lock(p->launch_mutex);
+    if (p->has_last && p->last_stream != st) CLEAR_CUDA_TRY(cudaStreamWaitEvent(st, p->ev_last, 0));
+    if (p->kernel == CLEAR_KERNEL_TCGEN05)
+        rc = launch_tc(*p, q, k, v, out, scale, st);
+    else if (p->kernel == CLEAR_KERNEL_TCGEN05_WS)
+        rc = launch_ws(*p, q, k, v, out, scale, st);
+    else
+        rc = launch_simt(*p, q, k, v, out, scale, st);
+    if (rc != CLEAR_OK) return rc;
+    CLEAR_CUDA_TRY(cudaEventRecord(p->ev_last, st));
+    p->last_stream = st;
+    p->has_last = true;
+    return CLEAR_OK;
 }
 
 // ---- plan cache of the unplanned entry points ----------------------------------------------------
@@ -253,7 +276,10 @@ struct CacheEntry {
     clear_plan_t *plan;
 };
 std::mutex g_cache_mutex;
-std::list<CacheEntry> g_cache;
+std::list<CacheEntry> g_cache;  // most recently used first
+// The cache keeps at most this many plans (CLEAR_CACHE_MAX_PLANS overrides it): a plan of the 8K workload owns
+// 211 MB of split-KV workspace.  The least recently used plan goes when a new shape arrives.
+constexpr int kMaxCachedPlans = 16;
 
 int cached_forward(const void *q, const void *k, const void *v, void *out, const Shape &shape, float scale, void *stream)
 {
@@ -267,19 +293,28 @@ int cached_forward(const void *q, const void *k, const void *v, void *out, const
     Shape s = shape;
     // the tensor-core kernel needs a positive scale; anything else goes to the CUDA-core kernel
     if (s.kernel == CLEAR_KERNEL_AUTO && !(scale > 0.f)) s.kernel = CLEAR_KERNEL_SIMT;
+    // The lock is held until the launch has been made: no other thread can evict or clear the plan while
+    // it is being launched (launches take microseconds).
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
     clear_plan_t *plan = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(g_cache_mutex);
-        for (const CacheEntry &e : g_cache)
-            if (e.device == dev && e.shape == s) {
-                plan = e.plan;
-                break;
-            }
-        if (!plan) {
-            rc = create_plan(&plan, s, false);
-            if (rc != CLEAR_OK) return rc;
-            g_cache.push_front(CacheEntry{s, dev, plan});
+    for (auto it = g_cache.begin(); it != g_cache.end(); ++it)
+        if (it->device == dev && it->shape == s) {
+            plan = it->plan;
+            g_cache.splice(g_cache.begin(), g_cache, it);
+            break;
         }
+    if (!plan) {
+        int cap = kMaxCachedPlans;
+        if (const char *e = std::getenv("CLEAR_CACHE_MAX_PLANS")) cap = std::max(1, std::atoi(e));
+        while ((int)g_cache.size() >= cap) {
+            // work of the evicted plan may still be in flight
+            if (cudaDeviceSynchronize() != cudaSuccess) (void)cudaGetLastError();
+            (void)clear_plan_destroy(g_cache.back().plan);
+            g_cache.pop_back();
+        }
+        rc = create_plan(&plan, s, false);
+        if (rc != CLEAR_OK) return rc;
+        g_cache.push_front(CacheEntry{s, dev, plan});
     }
     return forward(plan, q, k, v, out, scale, stream);
 }
@@ -474,9 +509,10 @@ int clear_plan_check(clear_plan_t *plan, void *stream)
     if (!plan) return CLEAR_ERR_INVALID_ARG;
     if (plan->host_only) return CLEAR_ERR_PLAN_MISMATCH;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    int status = 0;
-    CLEAR_CUDA_TRY(cudaMemcpyAsync(&status, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost, cs));
+    int words[kStatusWords] = {0, 0, 0, 0};
+    CLEAR_CUDA_TRY(cudaMemcpyAsync(words, plan->d_status, sizeof(words), cudaMemcpyDeviceToHost, cs));
     CLEAR_CUDA_TRY(cudaStreamSynchronize(cs));
+    const int status = words[3] != 0 ? words[3] : words[0];
     if (status != 0) {
         g_last_device_status = status;
         // a block that gave up may have left the work queue of the persistent kernel mid-way
@@ -485,6 +521,49 @@ int clear_plan_check(clear_plan_t *plan, void *stream)
         return CLEAR_ERR_DEVICE_TIMEOUT;
     }
     return CLEAR_OK;
+}
+
+int clear_cache_check(void *stream)
+{
+    int dev = -1;
+    CLEAR_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    int rc = CLEAR_OK;
+    for (CacheEntry &e : g_cache) {
+        if (e.device != dev) continue;
+        // the plan's last launch may have been made on another stream than the one given
+        if (e.plan->has_last && cudaEventSynchronize(e.plan->ev_last) != cudaSuccess) {
+            (void)cudaGetLastError();
+            if (rc == CLEAR_OK) rc = CLEAR_ERR_CUDA;
+        }
+        const int r = clear_plan_check(e.plan, stream);
+        if (r != CLEAR_OK && rc == CLEAR_OK) rc = r;
+    }
+    return rc;
+}
+
+int clear_plan_trim(clear_plan_t *plan)
+{
+    if (!plan) return CLEAR_ERR_INVALID_ARG;
+    if (plan->host_only) return CLEAR_OK;
+    int prev = -1;
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != plan->device) (void)cudaSetDevice(plan->device);
+    int rc = CLEAR_OK;
+    if (cudaDeviceSynchronize() != cudaSuccess) {
+        (void)cudaGetLastError();
+        rc = CLEAR_ERR_CUDA;
+    }
+    destroy_host_pipe(plan);
+    plan->pipe_decided = false;
+    for (void *&st : plan->d_stage) {
+        if (st && cudaFree(st) != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = CLEAR_ERR_CUDA;
+        }
+        st = nullptr;
+    }
+    if (prev >= 0 && prev != plan->device) (void)cudaSetDevice(prev);
+    return rc;
 }
 
 int clear_plan_destroy(clear_plan_t *plan)

@@ -40,10 +40,21 @@ struct clear_plan {
     clear_pair_item_t *d_pair_items = nullptr;
     clear_pair_step_t *d_pair_steps = nullptr;
     uint32_t *d_mask_table = nullptr;
-    // [0] status word: 0 = fine, set by a kernel whose bounded wait expired;
+    // [0] status word of the launch in flight: 0 = fine, set by a kernel whose bounded wait expired (the
+    //     rest of that launch's blocks then leave at once); the persistent kernel puts it back to zero when
+    //     its last block leaves;
     // [1] work-queue head and [2] finished-block count of the persistent kernel (both back at zero
-    // when a launch ends)
+    //     when a launch ends);
+    // [3] the first non-zero status of any launch since the last clear_plan_check (which reads and clears it)
     int *d_status = nullptr;
+
+    // Launches of one plan share its work queue, status words and split-KV workspace, so the library
+    // orders them on the device: a launch on another stream than the one before waits for that one's
+    // end (an event recorded behind every launch).
+    mutable std::mutex launch_mutex;
+    mutable cudaEvent_t ev_last = nullptr;
+    mutable cudaStream_t last_stream = nullptr;
+    mutable bool has_last = false;
 
     // split-KV workspace of the text-query rows (owned): per (bh, slot) 128 x head_dim fp32
     // un-normalised outputs, and per row the running maximum (log2 units) and the row sum
@@ -88,6 +99,11 @@ int launch_ws(const clear_plan &p, const void *q, const void *k, const void *v, 
               cudaStream_t stream);
 // Merge of the split-KV partial results of the text-query rows (both tensor-core kernels).
 int launch_text_combine(const clear_plan &p, void *out, cudaStream_t stream);
+
+// Tensor map (a CUtensorMap, 128 bytes) of a bf16 tensor of `rank` dims, innermost first, with 128-byte swizzle
+// and out-of-bounds elements read as zero; strides in bytes for dims 1..rank-1.  False if the driver refuses.
+bool encode_bf16_map(void *tensor_map, const void *base, int rank, const uint64_t *dims, const uint64_t *strides,
+                     const uint32_t *box);
 
 constexpr int kStatusWords = 4;
 

@@ -72,8 +72,8 @@ __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity)
     }
 }
 
-template <int D, bool P_SMEM>
-__global__ void __launch_bounds__(kThreads, P_SMEM ? 1 : 2)
+template <int D>
+__global__ void __launch_bounds__(kThreads, 2)
 clear_tc_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_constant__ CUtensorMap tm_k_img,
                 const __grid_constant__ CUtensorMap tm_v_img, const __grid_constant__ CUtensorMap tm_o_img,
                 const __grid_constant__ CUtensorMap tm_q_txt, const __grid_constant__ CUtensorMap tm_k_lin,
@@ -90,8 +90,7 @@ clear_tc_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
     const uint32_t sQ = smem_base, sK = sQ + kTileBytes, sV = sK + kTileBytes;
-    const uint32_t sP = sV + kTileBytes;  // only when P_SMEM
-    constexpr uint32_t kCtrlOff = (P_SMEM ? 3 * kTileBytes + 2 * kHalfBytes : 3 * kTileBytes);
+    constexpr uint32_t kCtrlOff = 3 * kTileBytes;
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(smem_gen + kCtrlOff);
     volatile int *abort_flag = &ctrl->abort_flag;
 
@@ -197,12 +196,7 @@ clear_tc_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint64_t bdesc = ptx::smem_desc_sw128(sV + kk * 2048, kHalfBytes, 1024);
                     const uint32_t acc = (i > 0 || kk > 0) ? 1u : 0u;
-                    if constexpr (P_SMEM) {
-                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                        ptx::mma_ss(tmem_O, ptx::smem_desc_sw128(sP + off, 16, 1024), bdesc, kIdescPV, acc);
-                    } else {
-                        ptx::mma_ts(tmem_O, tmem_S + kk * 8, bdesc, kIdescPV, acc);
-                    }
+                    ptx::mma_ts(tmem_O, tmem_S + kk * 8, bdesc, kIdescPV, acc);
                 }
                 ptx::tc_commit(b_o);
                 mma_pending = true;
@@ -333,23 +327,9 @@ clear_tc_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
                     l += p0 + p1;
                     pk[w >> 1][(w & 1) * 16 + (j >> 1)] = ptx::pack_bf16(p0, p1);
                 }
-            if constexpr (P_SMEM) {
-                // row r of the K-major, 128-byte-swizzled P tile: 16-byte chunk ch of half h
-                uint8_t *p_gen = smem_gen + (sP - smem_base);
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        uint4 val = make_uint4(pk[h][4 * ch], pk[h][4 * ch + 1], pk[h][4 * ch + 2], pk[h][4 * ch + 3]);
-                        *reinterpret_cast<uint4 *>(p_gen + h * kHalfBytes + r * 128 + ((ch ^ (r & 7)) << 4)) = val;
-                    }
-                ptx::fence_proxy_async_smem();
-                ptx::tmem_wait_st();
-            } else {
-                ptx::tmem_st32(tmem_S + lane_off, pk[0]);
-                ptx::tmem_st32(tmem_S + lane_off + 32, pk[1]);
-                ptx::tmem_wait_st();
-            }
+            ptx::tmem_st32(tmem_S + lane_off, pk[0]);
+            ptx::tmem_st32(tmem_S + lane_off + 32, pk[1]);
+            ptx::tmem_wait_st();
             ptx::tc_fence_before();
             ptx::mbar_arrive(b_p);
         }
@@ -445,37 +425,6 @@ clear_tc_combine_kernel(const float *__restrict__ partial_o, const float *__rest
 }
 
 // ---- host side: tensor maps and launch ---------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = []() -> EncodeTiledFn {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// bf16 tensor of `rank` dims (innermost first); strides in bytes for dims 1..rank-1.
-bool encode(CUtensorMap *tm, const void *base, int rank, const uint64_t *dims, const uint64_t *strides,
-            const uint32_t *box)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base),
-                     reinterpret_cast<const cuuint64_t *>(dims), reinterpret_cast<const cuuint64_t *>(strides),
-                     reinterpret_cast<const cuuint32_t *>(box), ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return rc == CUDA_SUCCESS;
-}
-
 int build_maps(const clear_plan &p, const void *q, const void *k, const void *v, void *out)
 {
     const Shape &s = p.shape;
@@ -490,44 +439,35 @@ int build_maps(const clear_plan &p, const void *q, const void *k, const void *v,
     const uint32_t box4[4] = {64, (uint32_t)kTileW, (uint32_t)kTileH, 1};
     for (int t = 0; t < 4; ++t) {
         const char *base = static_cast<const char *>(ptrs[t]) + T * row_b;
-        if (!encode(&tm[t], base, 4, dims4, str4, box4)) return CLEAR_ERR_CUDA;
+        if (!encode_bf16_map(&tm[t], base, 4, dims4, str4, box4)) return CLEAR_ERR_CUDA;
     }
     // token sequence as [BH][N][d] (K, V) and its text prefix [BH][n_text][d] (Q, O of text tiles)
     const uint64_t dims3[3] = {d, N, BH};
     const uint64_t dims3t[3] = {d, T > 0 ? T : 1, BH};
     const uint64_t str3[2] = {row_b, N * row_b};
     const uint32_t box3[3] = {64, (uint32_t)kTileTokens, 1};
-    if (!encode(&tm[4], q, 3, dims3t, str3, box3)) return CLEAR_ERR_CUDA;
-    if (!encode(&tm[5], k, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
-    if (!encode(&tm[6], v, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
-    if (!encode(&tm[7], out, 3, dims3t, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode_bf16_map(&tm[4], q, 3, dims3t, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode_bf16_map(&tm[5], k, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode_bf16_map(&tm[6], v, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode_bf16_map(&tm[7], out, 3, dims3t, str3, box3)) return CLEAR_ERR_CUDA;
     for (int t = 0; t < 4; ++t) p.tm_ptrs[t] = ptrs[t];
     p.tm_valid = true;
     return CLEAR_OK;
 }
 
-bool use_p_smem()
-{
-    static const bool v = []() {
-        const char *e = getenv("CLEAR_TC_P_SMEM");
-        return e && e[0] == '1';
-    }();
-    return v;
-}
-
-template <int D, bool P_SMEM>
+template <int D>
 int launch_variant(const clear_plan &p, const CUtensorMap *tm, const TcParams &prm, void *out, cudaStream_t stream)
 {
     const Shape &s = p.shape;
-    constexpr size_t kSmem = 1024 + 3 * (size_t)(D / 64) * 16384 + (P_SMEM ? 32768 : 0) + sizeof(Ctrl) + 64;
+    constexpr size_t kSmem = 1024 + 3 * (size_t)(D / 64) * 16384 + sizeof(Ctrl) + 64;
     static bool configured[64] = {};  // the attribute is set once per device
     if (p.device >= 0 && p.device < 64 && !configured[p.device]) {
-        CLEAR_CUDA_TRY(cudaFuncSetAttribute(clear_tc_kernel<D, P_SMEM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        CLEAR_CUDA_TRY(cudaFuncSetAttribute(clear_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)kSmem));
         configured[p.device] = true;
     }
     dim3 grid((unsigned)p.sch.items.size(), (unsigned)(s.B * s.H));
-    clear_tc_kernel<D, P_SMEM><<<grid, kThreads, kSmem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], tm[7],
+    clear_tc_kernel<D><<<grid, kThreads, kSmem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], tm[7],
                                                                   prm);
     CLEAR_CUDA_TRY(cudaGetLastError());
     return launch_text_combine(p, out, stream);
@@ -582,11 +522,8 @@ int launch_tc(const clear_plan &p, const void *q, const void *k, const void *v, 
     prm.partial_ml = p.d_partial_ml;
     prm.n_partial_slots = p.sch.n_partial_slots;
     prm.status = p.d_status;
-    const bool ps = use_p_smem();
-    if (p.shape.head_dim == 128)
-        return ps ? launch_variant<128, true>(p, tm, prm, out, stream) : launch_variant<128, false>(p, tm, prm, out, stream);
-    if (p.shape.head_dim == 64)
-        return ps ? launch_variant<64, true>(p, tm, prm, out, stream) : launch_variant<64, false>(p, tm, prm, out, stream);
+    if (p.shape.head_dim == 128) return launch_variant<128>(p, tm, prm, out, stream);
+    if (p.shape.head_dim == 64) return launch_variant<64>(p, tm, prm, out, stream);
     return CLEAR_ERR_UNSUPPORTED;
 }
 

@@ -74,7 +74,7 @@ struct WsParams {
     float *partial_ml;
     int n_partial_slots;
     __nv_bfloat16 *out;
-    int *status;  // [0] status word, [1] queue head, [2] finished blocks
+    int *status;  // [0] status word of this launch, [1] queue head, [2] finished blocks, [3] status kept for the host
 };
 
 struct Ctrl {
@@ -201,6 +201,16 @@ __device__ __forceinline__ int step_tile_index(int flags, int side)
     return (flags & CLEAR_STEP_USE0) ? 1 : 0;
 }
 
+// The last block of a launch to leave: the work queue goes back to zero, and a status some block raised
+// moves to the word that stays until the host has read it, so that the next launch starts clean.
+__device__ __forceinline__ void close_launch(int *status)
+{
+    atomicExch(status + 1, 0);
+    atomicExch(status + 2, 0);
+    const int raised = atomicExch(status, 0);
+    if (raised != 0) atomicCAS(status + 3, 0, raised);
+}
+
 template <int D>
 __global__ void __launch_bounds__(kWsThreads, 1)
 clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_constant__ CUtensorMap tm_k_img,
@@ -240,10 +250,7 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
         if (tid == 0) {
             // keep the finished-block count right so that the queue is reset for the next launch
             const int done = atomicAdd(prm.status + 2, 1);
-            if (done == (int)gridDim.x - 1) {
-                atomicExch(prm.status + 1, 0);
-                atomicExch(prm.status + 2, 0);
-            }
+            if (done == (int)gridDim.x - 1) close_launch(prm.status);
         }
         return;
     }
@@ -820,45 +827,11 @@ clear_ws_kernel(const __grid_constant__ CUtensorMap tm_q_img, const __grid_const
     if (tid == 0) {
         // the last block to finish puts the queue back to zero for the next launch
         const int done = atomicAdd(prm.status + 2, 1);
-        if (done == (int)gridDim.x - 1) {
-            atomicExch(prm.status + 1, 0);
-            atomicExch(prm.status + 2, 0);
-        }
+        if (done == (int)gridDim.x - 1) close_launch(prm.status);
     }
 }
 
 // ---- host side: tensor maps and launch ---------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = []() -> EncodeTiledFn {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// bf16 tensor of `rank` dims (innermost first); strides in bytes for dims 1..rank-1.
-bool encode(CUtensorMap *tm, const void *base, int rank, const uint64_t *dims, const uint64_t *strides,
-            const uint32_t *box)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    CUresult rc = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base),
-                     reinterpret_cast<const cuuint64_t *>(dims), reinterpret_cast<const cuuint64_t *>(strides),
-                     reinterpret_cast<const cuuint32_t *>(box), ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return rc == CUDA_SUCCESS;
-}
-
 // Maps 0..2: image part of q, k, v as [BH][grid_h][grid_w][d]; 3: text prefix of q as [BH][n_text][d];
 // 4, 5: k, v as the token sequence [BH][N][d].
 int build_maps(const clear_plan &p, const void *q, const void *k, const void *v)
@@ -874,15 +847,15 @@ int build_maps(const clear_plan &p, const void *q, const void *k, const void *v)
     const uint32_t box4[4] = {64, (uint32_t)kTileW, (uint32_t)kTileH, 1};
     for (int t = 0; t < 3; ++t) {
         const char *base = static_cast<const char *>(ptrs[t]) + T * row_b;
-        if (!encode(&tm[t], base, 4, dims4, str4, box4)) return CLEAR_ERR_CUDA;
+        if (!encode_bf16_map(&tm[t], base, 4, dims4, str4, box4)) return CLEAR_ERR_CUDA;
     }
     const uint64_t dims3[3] = {d, N, BH};
     const uint64_t dims3t[3] = {d, T > 0 ? T : 1, BH};
     const uint64_t str3[2] = {row_b, N * row_b};
     const uint32_t box3[3] = {64, (uint32_t)kTileTokens, 1};
-    if (!encode(&tm[3], q, 3, dims3t, str3, box3)) return CLEAR_ERR_CUDA;
-    if (!encode(&tm[4], k, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
-    if (!encode(&tm[5], v, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode_bf16_map(&tm[3], q, 3, dims3t, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode_bf16_map(&tm[4], k, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
+    if (!encode_bf16_map(&tm[5], v, 3, dims3, str3, box3)) return CLEAR_ERR_CUDA;
     for (int t = 0; t < 3; ++t) p.tm_ptrs[t] = ptrs[t];
     p.tm_ptrs[3] = nullptr;
     p.tm_valid = true;

@@ -427,3 +427,154 @@ def test_host_tensor_entry_point_in_chunks(B, H, monkeypatch):
     want = oracle.attn(q[:1, :2], k[:1, :2], v[:1, :2], gh, gw, T, r, scale)
     assert_close_bf16(oh[:1, :2], want, "chunked host entry point")
     plan.destroy()
+
+
+# ----------------------------------------------------------------------------------------------
+# the mask at full size: every row, every border class the real schedules produce
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("gh,gw,T,r", [(128, 128, 512, 16.0), (192, 320, 512, 16.0)], ids=["c2", "c3_192x320"])
+def test_mask_is_exact_on_every_row_at_full_size(gh, gw, T, r):
+    """Q = 0 makes every allowed key weigh the same, so the output reads the mask back: column 0 of V marks
+    the text keys (out = n_text / count_i on EVERY row, against the oracle's all-pairs count of Eq. 3), column 1
+    is all ones (out = 1), and each further column is 1 on one planted key only -- grid corners, borders, tile
+    seams, random positions -- so that out is 1 / count_i where Eq. 3 allows that key and exactly 0 elsewhere
+    (the oracle's mask row of the key, the mask being symmetric).  A wrong bit in any mask-table entry or
+    clipped border patch moves many such pairs."""
+    d, N = 128, T + gh * gw
+    _, counts = oracle.mask_counts(gh, gw, T, r)
+    rng = np.random.default_rng(gh * 7 + gw)
+    ys = sorted({0, 7, 8, 15, 16, gh // 2 - 1, gh // 2, gh - 17, gh - 16, gh - 9, gh - 8, gh - 1} & set(range(gh)))
+    xs = sorted({0, 15, 16, 31, 32, gw // 2 - 1, gw // 2, gw - 33, gw - 32, gw - 17, gw - 16, gw - 1} & set(range(gw)))
+    planted = [T + y * gw + x for y in ys for x in xs][: d - 2 - 24]
+    planted += [int(T + p) for p in rng.integers(0, gh * gw, 20)] + [0, T // 2, T - 1, T]
+    planted = planted[: d - 2]
+    v = torch.zeros(1, 1, N, d, dtype=torch.float32)
+    v[0, 0, :T, 0] = 1.0
+    v[0, 0, :, 1] = 1.0
+    for c, j in enumerate(planted):
+        v[0, 0, j, 2 + c] = 1.0
+    v = v.to(torch.bfloat16)
+    g = torch.Generator(device="cpu").manual_seed(3)
+    k = torch.randn(1, 1, N, d, generator=g).to(torch.bfloat16)
+    q = torch.zeros(1, 1, N, d, dtype=torch.bfloat16)
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    out = torch.full_like(qd, float("nan"))
+    clear.clear_attn_fwd(qd, kd, vd, out, gh, gw, T, r, 1 / math.sqrt(d))
+    torch.cuda.synchronize()
+    clear.clear_cache_check()
+    got = out[0, 0].cpu().double().numpy()
+    assert np.isfinite(got).all()
+    inv = 1.0 / counts.astype(np.float64)
+    # bf16 output: half a unit in the last place is 2^-9 relative
+    np.testing.assert_allclose(got[:, 0], T * inv, rtol=4e-3, atol=0)
+    np.testing.assert_allclose(got[:, 1], 1.0, rtol=4e-3, atol=0)
+    for c, j in enumerate(planted):
+        allowed = oracle.mask_row(j, gh, gw, T, r).astype(bool)   # column j of M = row j (M is symmetric)
+        col = got[:, 2 + c]
+        assert (col[~allowed] == 0.0).all(), f"planted key {j}: weight outside the window"
+        np.testing.assert_allclose(col[allowed], inv[allowed], rtol=4e-3, atol=0, err_msg=f"planted key {j}")
+    clear.clear_cache_clear()
+
+
+@pytest.mark.parametrize("kernel", [clear.KERNEL_SIMT] + TC_KERNELS, ids=["simt"] + TC_IDS)
+@pytest.mark.parametrize("r", [math.sqrt(2.0), math.sqrt(5.0)])
+def test_radii_that_fp32_cannot_hold_exactly(kernel, r):
+    """The C ABI takes the radius as a float: sqrt(2) becomes 1.41421354, whose square is below 2, so the
+    diagonal neighbours (d^2 = 2) are NOT allowed (threshold ceil(r^2) = 2), while the double sqrt(2) would allow
+    them.  Both sides get the fp32 value."""
+    r32 = float(np.float32(r))
+    gh, gw, T, d = 13, 19, 7, 128
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=int(r * 1000))
+    scale = 1 / math.sqrt(d)
+    want = oracle.attn(q, k, v, gh, gw, T, r32, scale)
+    got = run_plan(q, k, v, gh, gw, T, r32, scale, kernel)
+    assert_close_bf16(got, want, f"radius {r32}")
+
+
+# ----------------------------------------------------------------------------------------------
+# streams, and the error path of a kernel that gave up (no wait is made to expire)
+# ----------------------------------------------------------------------------------------------
+def test_one_shape_from_two_streams_at_once():
+    """Calls of clear_attn_fwd for one shape share a cached plan; the library orders them on the device, so two
+    streams may issue them back to back with different tensors."""
+    gh, gw, T, r, d, H = 64, 64, 200, 8.0, 128, 4
+    scale = 1 / math.sqrt(d)
+    ins = [[t.to(dev()) for t in workloads.make_custom(1, H, gh, gw, T, d, seed=900 + i)] for i in range(2)]
+    want = []
+    for qd, kd, vd in ins:
+        o = torch.full_like(qd, float("nan"))
+        clear.clear_attn_fwd(qd, kd, vd, o, gh, gw, T, r, scale)
+        torch.cuda.synchronize()
+        want.append(o)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [torch.full_like(ins[i][0], float("nan")) for i in range(2)]
+    torch.cuda.synchronize()
+    for rep in range(6):
+        for i in (0, 1):
+            qd, kd, vd = ins[i]
+            clear.clear_attn_fwd(qd, kd, vd, outs[i], gh, gw, T, r, scale, stream=streams[i])
+    for s in streams:
+        s.synchronize()
+    clear.clear_cache_check()
+    for i in (0, 1):
+        assert torch.equal(outs[i], want[i])
+    rows = np.array([(0, h, i) for h in (0, H - 1) for i in (0, T - 1, T, T + 65, T + gh * gw - 1)], dtype=np.int64)
+    q, k, v = (t.cpu() for t in ins[1])
+    ref = oracle.attn_rows(q, k, v, gh, gw, T, r, scale, rows)
+    assert_close_bf16(outs[1].cpu()[rows[:, 0], rows[:, 1], rows[:, 2]], ref, "two streams")
+    clear.clear_cache_clear()
+
+
+@pytest.mark.parametrize("cached", [False, True], ids=["planned", "cached"])
+def test_a_launch_that_finds_the_status_word_raised_is_reported_and_the_next_one_runs(cached, monkeypatch):
+    """The plan is created with its status word preset, as if a block's bounded wait had expired: the first
+    launch takes the early-leave path (every block returns at once, the last one puts the work queue back),
+    the check reports DEVICE_TIMEOUT with the preset code, and the launch after that is correct."""
+    gh, gw, T, r, d = 24, 40, 130, 8.0, 128
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=31)
+    scale = 1 / math.sqrt(d)
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    out = torch.full_like(qd, -3.0)
+    clear.clear_cache_clear()
+    monkeypatch.setenv("CLEAR_TEST_PRESET_STATUS", "77")
+    plan = None
+    if cached:
+        run = lambda o: clear.clear_attn_fwd(qd, kd, vd, o, gh, gw, T, r, scale)
+        check = clear.clear_cache_check
+    else:
+        plan = clear.Plan(1, 2, gh, gw, T, d, r, kernel=clear.KERNEL_TCGEN05_WS)
+        run = lambda o: plan.forward(qd, kd, vd, o, scale)
+        check = plan.check
+    run(out)                                   # the plan (and its preset status word) is made here when cached
+    monkeypatch.delenv("CLEAR_TEST_PRESET_STATUS")
+    with pytest.raises(clear.ClearError) as e:
+        check()
+    assert e.value.status == clear.ERR_DEVICE_TIMEOUT and clear.last_device_status() == 77
+    assert bool((out == -3.0).all()), "a launch that gave up must not write"
+    check()                                    # the record is cleared
+    out2 = torch.full_like(qd, float("nan"))
+    run(out2)
+    check()
+    want = oracle.attn(q, k, v, gh, gw, T, r, scale)
+    assert_close_bf16(out2.cpu(), want, "launch after a reported expiry")
+    if plan is not None:
+        plan.destroy()
+    clear.clear_cache_clear()
+
+
+def test_the_plan_cache_keeps_a_bounded_number_of_shapes(monkeypatch):
+    monkeypatch.setenv("CLEAR_CACHE_MAX_PLANS", "2")
+    clear.clear_cache_clear()
+    d, scale = 64, 0.125
+    free0 = torch.cuda.mem_get_info()[0]
+    outs = []
+    for gh in (8, 16, 24, 32, 8):              # five calls, four shapes, at most two plans alive
+        q, k, v = (t.to(dev()) for t in workloads.make_custom(1, 1, gh, 16, 5, d, seed=gh))
+        o = torch.full_like(q, float("nan"))
+        clear.clear_attn_fwd(q, k, v, o, gh, 16, 5, 3.0, scale)
+        outs.append((gh, q.cpu(), k.cpu(), v.cpu(), o))
+    torch.cuda.synchronize()
+    for gh, q, k, v, o in outs:
+        assert_close_bf16(o.cpu(), oracle.attn(q, k, v, gh, 16, 5, 3.0, scale), f"cached shape {gh}")
+    clear.clear_cache_clear()
+    del outs

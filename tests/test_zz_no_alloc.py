@@ -1,4 +1,4 @@
-"""The no-allocation entry point, `clear_attn_fwd_static`, against the planned entry point.
+"""The no-allocation entry point, `clear_attn_fwd_static`, against the planned entry points and the oracle.
 
 Some callers cannot allocate device memory where attention runs: a host that works inside a fixed,
 pre-partitioned memory budget, a plug-in whose embedding framework owns every device byte, a process whose
@@ -9,9 +9,11 @@ every other test; it must also pass alone in a fresh process.
 """
 import math
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import clear_oracle as oracle
 from paper_2412_16112_b200 import binding as clear
 from paper_2412_16112_b200 import workloads
 
@@ -36,13 +38,30 @@ def test_static_entry_point_matches_the_planned_one_twice_in_a_row():
     qd, kd, vd = (t.to(dev) for t in (q, k, v))
     want = torch.full_like(qd, float("nan"))
     clear.clear_attn_fwd(qd, kd, vd, want, gh, gw, T, r, scale)
+    # the same kernel through a plan of its own (cudaMalloc'ed tables and scratch): equal bit for bit
+    same = torch.full_like(qd, float("nan"))
+    plan = clear.Plan(1, 2, gh, gw, T, d, r, kernel=clear.KERNEL_TCGEN05)
+    plan.forward(qd, kd, vd, same, scale)
+    plan.check()
     torch.cuda.synchronize()
 
-    for _ in range(2):                                   # the second call reuses tables and dirty scratch
-        got = torch.full_like(qd, float("nan"))
-        clear.clear_attn_fwd_static(qd, kd, vd, got, gh, gw, T, r, scale)
-        torch.cuda.synchronize()
-        assert _close(got, want)
+    got = torch.full_like(qd, float("nan"))
+    clear.clear_attn_fwd_static(qd, kd, vd, got, gh, gw, T, r, scale)   # first call: set-up + table upload
+    torch.cuda.synchronize()
+    assert _close(got, want) and torch.equal(got, same)
+    # the second call reuses tables and dirty scratch, and the device's free memory does not move across it
+    got.fill_(float("nan"))
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    clear.clear_attn_fwd_static(qd, kd, vd, got, gh, gw, T, r, scale)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before, "the no-allocation entry point changed the free device memory"
+    assert _close(got, want) and torch.equal(got, same)
+    # and against the CPU oracle on sampled rows
+    rows = np.array([(0, h, i) for h in (0, 1) for i in (0, T - 1, T, T + 97, T + gh * gw // 2, T + gh * gw - 1)], dtype=np.int64)
+    ref = oracle.attn_rows(q, k, v, gh, gw, T, r, scale, rows)
+    err = np.abs(got.cpu()[rows[:, 0], rows[:, 1], rows[:, 2]].double().numpy() - ref)
+    assert err.max() <= BF16_MAX and err.mean() <= BF16_MEAN
 
     # another shape in between forces a table re-upload into the same array, then back again
     gh2, gw2, T2, r2 = 24, 40, 130, 8.0
@@ -55,7 +74,8 @@ def test_static_entry_point_matches_the_planned_one_twice_in_a_row():
     clear.clear_attn_fwd_static(qd, kd, vd, got, gh, gw, T, r, scale)
     torch.cuda.synchronize()
     assert _close(got2, want2)
-    assert _close(got, want)
+    assert _close(got, want) and torch.equal(got, same)
+    plan.destroy()
     clear.clear_cache_clear()
 
 
