@@ -164,6 +164,20 @@ int clear_attn_fwd_f32(const void *q, const void *k, const void *v, void *out, i
                        int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale,
                        void *stream);
 
+/* Backward pass of the operator for fp32 tensors (the distillation losses of Sec. 3.3, Eq. 4-6, reach the
+ * attention parameters through it): given the upstream gradient d_out of the output of clear_attn_fwd_f32,
+ *     p_ij  = softmax_j(scale q_i . k_j) over the keys Eq. 3 allows query i (Eq. 1),
+ *     dS_ij = p_ij (d_out_i . v_j - sum_j' p_ij' d_out_i . v_j'),
+ *     dq_i = scale sum_j dS_ij k_j,   dk_j = scale sum_i dS_ij q_i,   dv_j = sum_i p_ij d_out_i.
+ * All seven tensors are device pointers, [B, H, N, head_dim] contiguous fp32, 16-byte aligned; q, k, v,
+ * d_out are read, dq, dk, dv fully written (dk and dv are zeroed on `stream` first; sums into them are
+ * atomic, so their last bits depend on the order of arrival).  Nothing but `stream` is synchronised.
+ * A CUDA-core kernel meant for small problems (two atomic adds per channel of every allowed pair).
+ * Errors: INVALID_ARG, MISALIGNED, UNSUPPORTED (head_dim > 256), CUDA. */
+int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk,
+                       void *dv, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius,
+                       float scale, void *stream);
+
 /* Build the schedule for one shape on the current device (Eq. 3 turned into integer geometry):
  * the threshold ceil(radius^2), for every 2-D query patch the list of key patches that meet its
  * radius-r dilation (with a flag telling whether the exact mask is needed) plus the text tiles,

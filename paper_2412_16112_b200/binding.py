@@ -27,7 +27,7 @@ EXPORTS = [
     "clear_plan_tables", "clear_attn_fwd_planned", "clear_attn_fwd_host", "clear_plan_info",
     "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
     "clear_last_cuda_error", "clear_attn_fwd_static", "clear_plan_pair_tables",
-    "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim",
+    "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim", "clear_attn_bwd_f32",
 ]
 
 
@@ -90,6 +90,7 @@ def load() -> ctypes.CDLL:
         lib.clear_attn_fwd.argtypes = fwd_args
         lib.clear_attn_fwd_f32.argtypes = fwd_args
         lib.clear_attn_fwd_static.argtypes = fwd_args
+        lib.clear_attn_bwd_f32.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp]
         plan_args = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, f32, i32, i32]
         lib.clear_plan_create.argtypes = plan_args
         lib.clear_plan_create_host.argtypes = plan_args
@@ -169,6 +170,19 @@ def clear_attn_fwd(q, k, v, out, grid_h, grid_w, n_text, radius, scale, stream=N
     _check(load().clear_attn_fwd(*ptrs, B, H, grid_h, grid_w, n_text, d, float(radius), float(scale),
                                  _stream_ptr(stream)), "clear_attn_fwd")
     return out
+
+
+def clear_attn_bwd_f32(q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radius, scale, stream=None):
+    """fp32 backward pass: gradients of q, k, v into ``dq``, ``dk``, ``dv`` for the upstream gradient ``d_out``."""
+    import torch
+    for t in (q, k, v, d_out, dq, dk, dv):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.float32 and t.shape == q.shape):
+            raise ValueError("backward tensors must be contiguous fp32 CUDA tensors of one [B, H, N, d] shape")
+    B, H, _, d = q.shape
+    _check(load().clear_attn_bwd_f32(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_out.data_ptr(), dq.data_ptr(),
+                                     dk.data_ptr(), dv.data_ptr(), B, H, grid_h, grid_w, n_text, d, float(radius),
+                                     float(scale), _stream_ptr(stream)), "clear_attn_bwd_f32")
+    return dq, dk, dv
 
 
 def clear_attn_fwd_f32(q, k, v, out, grid_h, grid_w, n_text, radius, scale, stream=None):

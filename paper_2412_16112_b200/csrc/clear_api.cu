@@ -281,20 +281,13 @@ std::list<CacheEntry> g_cache;  // most recently used first
 // 211 MB of split-KV workspace.  The least recently used plan goes when a new shape arrives.
 constexpr int kMaxCachedPlans = 16;
 
-int cached_forward(const void *q, const void *k, const void *v, void *out, const Shape &shape, float scale, void *stream)
+// Finds (or makes) the cached plan of a shape on the current device and calls `launch(plan)` with the cache
+// locked: no other thread can evict or clear the plan while it is being launched (launches take microseconds).
+template <typename Launch>
+int with_cached_plan(const Shape &s, Launch &&launch)
 {
-    int rc = validate_shape(shape);
-    if (rc != CLEAR_OK) return rc;
-    if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
-    rc = check_tensors(q, k, v, out);
-    if (rc != CLEAR_OK) return rc;
     int dev = -1;
     CLEAR_CUDA_TRY(cudaGetDevice(&dev));
-    Shape s = shape;
-    // the tensor-core kernel needs a positive scale; anything else goes to the CUDA-core kernel
-    if (s.kernel == CLEAR_KERNEL_AUTO && !(scale > 0.f)) s.kernel = CLEAR_KERNEL_SIMT;
-    // The lock is held until the launch has been made: no other thread can evict or clear the plan while
-    // it is being launched (launches take microseconds).
     std::lock_guard<std::mutex> lock(g_cache_mutex);
     clear_plan_t *plan = nullptr;
     for (auto it = g_cache.begin(); it != g_cache.end(); ++it)
@@ -312,11 +305,24 @@ int cached_forward(const void *q, const void *k, const void *v, void *out, const
             (void)clear_plan_destroy(g_cache.back().plan);
             g_cache.pop_back();
         }
-        rc = create_plan(&plan, s, false);
+        const int rc = create_plan(&plan, s, false);
         if (rc != CLEAR_OK) return rc;
         g_cache.push_front(CacheEntry{s, dev, plan});
     }
-    return forward(plan, q, k, v, out, scale, stream);
+    return launch(plan);
+}
+
+int cached_forward(const void *q, const void *k, const void *v, void *out, const Shape &shape, float scale, void *stream)
+{
+    int rc = validate_shape(shape);
+    if (rc != CLEAR_OK) return rc;
+    if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
+    rc = check_tensors(q, k, v, out);
+    if (rc != CLEAR_OK) return rc;
+    Shape s = shape;
+    // the tensor-core kernel needs a positive scale; anything else goes to the CUDA-core kernel
+    if (s.kernel == CLEAR_KERNEL_AUTO && !(scale > 0.f)) s.kernel = CLEAR_KERNEL_SIMT;
+    return with_cached_plan(s, [&](clear_plan_t *plan) { return forward(plan, q, k, v, out, scale, stream); });
 }
 
 }  // namespace
@@ -338,6 +344,22 @@ int clear_attn_fwd_f32(const void *q, const void *k, const void *v, void *out, i
 {
     Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, CLEAR_F32, CLEAR_KERNEL_SIMT};
     return cached_forward(q, k, v, out, s, scale, stream);
+}
+
+int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk, void *dv,
+                       int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale,
+                       void *stream)
+{
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, CLEAR_F32, CLEAR_KERNEL_SIMT};
+    int rc = validate_shape(s);
+    if (rc != CLEAR_OK) return rc;
+    if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
+    rc = check_tensors(q, k, v, d_out);
+    if (rc == CLEAR_OK) rc = check_tensors(dq, dk, dv, dq);
+    if (rc != CLEAR_OK) return rc;
+    return with_cached_plan(s, [&](clear_plan_t *plan) {
+        return launch_bwd_f32(*plan, q, k, v, d_out, dq, dk, dv, scale, static_cast<cudaStream_t>(stream));
+    });
 }
 
 int clear_plan_create(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text, int head_dim,

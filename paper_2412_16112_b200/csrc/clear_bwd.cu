@@ -1,0 +1,162 @@
+// Backward pass of the CLEAR attention operator on the CUDA cores, fp32 throughout: dQ, dK, dV for an
+// upstream gradient dO of  O = softmax(scale Q K^T + log M) V  (Eq. 1 under the mask of Eq. 3), the step
+// through which the distillation losses of Sec. 3.3 (Eq. 4-6) reach the attention parameters.
+//
+// One warp per query, lanes split the head dimension, keys walked as in the forward CUDA-core kernel (the
+// text tokens, then per grid row within reach the clipped run of columns).  Two sweeps over the allowed keys:
+//   1. online softmax: row maximum m, row sum l, the un-normalised output, hence delta = dO . O;
+//   2. per key: p = exp(s - m) / l, dP = dO . v, dS = p (dP - delta);  dQ += scale dS k  (registers),
+//      dK_j += scale dS q  and  dV_j += p dO  (atomic adds: several queries share a key).
+// Sized for small problems (the fp32 configuration): 2 d atomic adds per allowed pair.
+#include "clear_internal.hpp"
+
+namespace clear {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+template <int EPL>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+clear_bwd_kernel(const float *__restrict__ q, const float *__restrict__ k, const float *__restrict__ v,
+                 const float *__restrict__ d_out, float *__restrict__ dq, float *dk, float *dv, int grid_h, int grid_w,
+                 int n_text, int d, const int32_t *__restrict__ half_width, int n_half_width, float scale)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t N = (int64_t)n_text + (int64_t)grid_h * grid_w;
+    const int64_t i = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (i >= N) return;  // whole warp leaves together
+    const int64_t base = (int64_t)blockIdx.y * N * d;
+
+    float qv[EPL], gv[EPL], acc[EPL];
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) {
+        const int e = lane + 32 * t;
+        qv[t] = e < d ? q[base + i * d + e] : 0.f;
+        gv[t] = e < d ? d_out[base + i * d + e] : 0.f;
+        acc[t] = 0.f;
+    }
+    auto dot_row = [&](const float (&a)[EPL], const float *__restrict__ rows, int64_t j) {
+        float part = 0.f;
+#pragma unroll
+        for (int t = 0; t < EPL; ++t) {
+            const int e = lane + 32 * t;
+            if (e < d) part = fmaf(a[t], rows[base + j * d + e], part);
+        }
+        return warp_sum(part);
+    };
+    // the keys Eq. 3 allows this query, as runs of consecutive tokens
+    auto for_each_run = [&](auto &&body) {
+        if (i < n_text) {
+            body((int64_t)0, N);
+            return;
+        }
+        body((int64_t)0, (int64_t)n_text);
+        const int64_t pix = i - n_text;
+        const int y = (int)(pix / grid_w), x = (int)(pix % grid_w);
+        const int R = n_half_width - 1;
+        for (int dy = -R; dy <= R; ++dy) {
+            const int yy = y + dy;
+            if (yy < 0 || yy >= grid_h) continue;
+            const int hw = half_width[dy < 0 ? -dy : dy];
+            const int lo = max(x - hw, 0), hi = min(x + hw, grid_w - 1);
+            const int64_t row0 = (int64_t)n_text + (int64_t)yy * grid_w;
+            body(row0 + lo, row0 + hi + 1);
+        }
+    };
+
+    // ---- sweep 1: m, l and the un-normalised output ------------------------------------------------
+    float m = -INFINITY, l = 0.f;
+    for_each_run([&](int64_t j0, int64_t j1) {
+        for (int64_t j = j0; j < j1; ++j) {
+            const float s = scale * dot_row(qv, k, j);
+            const float m_new = fmaxf(m, s);
+            const float alpha = expf(m - m_new);  // m = -inf at the first key: alpha = 0
+            const float p = expf(s - m_new);
+            l = l * alpha + p;
+#pragma unroll
+            for (int t = 0; t < EPL; ++t) {
+                const int e = lane + 32 * t;
+                if (e < d) acc[t] = fmaf(p, v[base + j * d + e], acc[t] * alpha);
+            }
+            m = m_new;
+        }
+    });
+    const float inv_l = 1.f / l;  // l >= 1: the query itself (image) or any token (text) is always allowed
+    float part = 0.f;
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) part = fmaf(gv[t], acc[t], part);
+    const float delta = warp_sum(part) * inv_l;  // dO . O = sum_j p_ij dP_ij
+
+    // ---- sweep 2: the gradients --------------------------------------------------------------------
+    float gq[EPL];
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) gq[t] = 0.f;
+    for_each_run([&](int64_t j0, int64_t j1) {
+        for (int64_t j = j0; j < j1; ++j) {
+            const float p = expf(scale * dot_row(qv, k, j) - m) * inv_l;
+            const float ds = p * (dot_row(gv, v, j) - delta) * scale;
+#pragma unroll
+            for (int t = 0; t < EPL; ++t) {
+                const int e = lane + 32 * t;
+                if (e < d) {
+                    gq[t] = fmaf(ds, k[base + j * d + e], gq[t]);
+                    atomicAdd(dk + base + j * d + e, ds * qv[t]);
+                    atomicAdd(dv + base + j * d + e, p * gv[t]);
+                }
+            }
+        }
+    });
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) {
+        const int e = lane + 32 * t;
+        if (e < d) dq[base + i * d + e] = gq[t];
+    }
+}
+
+}  // namespace
+
+int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq,
+                   void *dk, void *dv, float scale, cudaStream_t stream)
+{
+    const Shape &s = p.shape;
+    const int64_t N = (int64_t)s.n_text + (int64_t)s.grid_h * s.grid_w;
+    const size_t bytes = (size_t)s.B * s.H * N * s.head_dim * sizeof(float);
+    // several queries add into one key's gradients: they start at zero
+    CLEAR_CUDA_TRY(cudaMemsetAsync(dk, 0, bytes, stream));
+    CLEAR_CUDA_TRY(cudaMemsetAsync(dv, 0, bytes, stream));
+    dim3 grid((unsigned)((N + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)(s.B * s.H));
+    dim3 block(kWarpsPerBlock * 32);
+    const int n_hw = (int)p.sch.half_width.size();
+    const int epl = (s.head_dim + 31) / 32;
+#define CLEAR_BWD_CASE(E)                                                                                            \
+    case E:                                                                                                          \
+        clear_bwd_kernel<E><<<grid, block, 0, stream>>>((const float *)q, (const float *)k, (const float *)v,       \
+                                                        (const float *)d_out, (float *)dq, (float *)dk, (float *)dv, \
+                                                        s.grid_h, s.grid_w, s.n_text, s.head_dim, p.d_half_width,    \
+                                                        n_hw, scale);                                                \
+        break;
+    switch (epl) {
+        CLEAR_BWD_CASE(1)
+        CLEAR_BWD_CASE(2)
+        CLEAR_BWD_CASE(3)
+        CLEAR_BWD_CASE(4)
+        CLEAR_BWD_CASE(5)
+        CLEAR_BWD_CASE(6)
+        CLEAR_BWD_CASE(7)
+        CLEAR_BWD_CASE(8)
+        default:
+            return CLEAR_ERR_UNSUPPORTED;
+    }
+#undef CLEAR_BWD_CASE
+    CLEAR_CUDA_TRY(cudaGetLastError());
+    return CLEAR_OK;
+}
+
+}  // namespace clear

@@ -97,6 +97,9 @@ int launch_tc(const clear_plan &p, const void *q, const void *k, const void *v, 
               cudaStream_t stream);
 int launch_ws(const clear_plan &p, const void *q, const void *k, const void *v, void *out, float scale,
               cudaStream_t stream);
+// fp32 backward pass on the CUDA cores (dk and dv are zeroed on the stream first).
+int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq,
+                   void *dk, void *dv, float scale, cudaStream_t stream);
 // Merge of the split-KV partial results of the text-query rows (both tensor-core kernels).
 int launch_text_combine(const clear_plan &p, void *out, cudaStream_t stream);
 

@@ -1,0 +1,55 @@
+"""GPU parity of the backward pass (`clear_attn_bwd_f32`, through the C ABI) against its fp64 CPU oracle,
+element by element on small shapes."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import clear_oracle_bwd as oracle_bwd
+from paper_2412_16112_b200 import binding as clear
+from paper_2412_16112_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+# fp32 arithmetic with fp32 atomic sums of up to a few hundred terms of order one
+BWD_ATOL = 1e-4
+
+
+@pytest.mark.parametrize("gh,gw,T,r,d", [
+    (16, 16, 16, 4.0, 64),      # the tiny fp32 configuration
+    (13, 19, 7, 4.0, 128),      # ragged on both axes
+    (8, 16, 0, 1.0, 128),       # no text, self only: dv = d_out, dq = dk = 0
+    (9, 33, 0, 5.5, 40),        # head size that is no multiple of 32, non-integer radius
+    (20, 50, 3, 100.0, 64),     # radius beyond the diagonal: full attention
+    (1, 70, 2, 3.0, 96),        # single-row grid
+    (24, 40, 130, 8.0, 64),
+])
+def test_backward_matches_the_oracle_everywhere(gh, gw, T, r, d):
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, dtype="f32", qk_norm=False, seed=gh * 31 + gw)
+    g = torch.Generator(device="cpu").manual_seed(gh + gw)
+    d_out = torch.randn(q.shape, generator=g, dtype=torch.float32)
+    scale = 1 / math.sqrt(d)
+    want = oracle_bwd.attn_bwd(q, k, v, d_out, gh, gw, T, r, scale)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, gd = (t.to(dev) for t in (q, k, v, d_out))
+    dq, dk, dv = (torch.full_like(qd, float("nan")) for _ in range(3))
+    for _ in range(2):      # the second call finds dk, dv dirty and must start them at zero again
+        clear.clear_attn_bwd_f32(qd, kd, vd, gd, dq, dk, dv, gh, gw, T, r, scale)
+    torch.cuda.synchronize()
+    for name, got, ref in (("dq", dq, want[0]), ("dk", dk, want[1]), ("dv", dv, want[2])):
+        err = np.abs(got.cpu().double().numpy() - ref)
+        assert np.isfinite(err).all(), f"{name}: non-finite"
+        assert err.max() <= BWD_ATOL, f"{name}: max {err.max():.3e}"
+    clear.clear_cache_clear()
+
+
+def test_backward_argument_errors():
+    dev = torch.device("cuda:0")
+    x = torch.zeros(1, 1, 272, 64, device=dev)
+    p = x.data_ptr()
+    lib = clear.load()
+    assert lib.clear_attn_bwd_f32(p, p, p, p, p, p, p, 1, 1, 16, 16, 16, 64, 0.0, 0.125, None) == clear.ERR_INVALID_ARG
+    assert lib.clear_attn_bwd_f32(p, p, p, None, p, p, p, 1, 1, 16, 16, 16, 64, 4.0, 0.125, None) == clear.ERR_INVALID_ARG
+    assert lib.clear_attn_bwd_f32(p, p, p, p, p, p + 4, p, 1, 1, 16, 16, 16, 64, 4.0, 0.125, None) == clear.ERR_MISALIGNED
+    assert lib.clear_attn_bwd_f32(p, p, p, p, p, p, p, 1, 1, 16, 16, 16, 64, 4.0, float("nan"), None) == clear.ERR_INVALID_ARG
