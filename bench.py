@@ -13,6 +13,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -44,28 +45,81 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons for one GPU while the timed region runs."""
+    """Samples SM clocks and throttle reasons of one GPU while the timed region runs (read-only queries):
+    through NVML every 20 ms where the Python binding is there, else through nvidia-smi (slower per sample)."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
+    PERIOD_S = 0.02
 
     def __init__(self, index: int):
         self.index = index
-        self.samples = []
+        self.sm, self.mx, self.power = [], [], []
+        self.reasons = set()
+        self.source = "nvidia-smi"
         self._stop = threading.Event()
         self._thread = threading.Thread(target=self._run, daemon=True)
+        self._nvml = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible:
+                ids = [x.strip() for x in visible.split(",") if x.strip()]
+                if index < len(ids) and ids[index].isdigit():
+                    phys = int(ids[index])
+            self._handle = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self._nvml = pynvml
+            self.source = "nvml"
+        except Exception:
+            self._nvml = None
+
+    def _sample_nvml(self):
+        n = self._nvml
+        self.sm.append(float(n.nvmlDeviceGetClockInfo(self._handle, n.NVML_CLOCK_SM)))
+        self.mx.append(float(n.nvmlDeviceGetMaxClockInfo(self._handle, n.NVML_CLOCK_SM)))
+        try:
+            self.power.append(n.nvmlDeviceGetPowerUsage(self._handle) / 1000.0)
+        except Exception:
+            pass
+        try:
+            bits = n.nvmlDeviceGetCurrentClocksEventReasons(self._handle)
+        except Exception:
+            bits = n.nvmlDeviceGetCurrentClocksThrottleReasons(self._handle)
+        for name, const in (("hw_slowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                            ("hw_thermal_slowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                            ("sw_thermal_slowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                            ("sw_power_cap", "nvmlClocksThrottleReasonSwPowerCap")):
+            if bits & getattr(n, const, 0):
+                self.reasons.add(name)
+
+    def _sample_smi(self):
+        out = subprocess.run(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                              "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+        parts = [x.strip() for x in out.strip().split(",")]
+        if len(parts) < 7:
+            return
+        self.sm.append(float(parts[0]))
+        self.mx.append(float(parts[1]))
+        try:
+            self.power.append(float(parts[2]))
+        except ValueError:
+            pass
+        for name, val in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], parts[3:7]):
+            if val.lower().startswith("active"):
+                self.reasons.add(name)
 
     def _run(self):
         while not self._stop.is_set():
             try:
-                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
-                parts = [x.strip() for x in out.strip().split(",")]
-                if len(parts) >= 7:
-                    self.samples.append(parts)
+                if self._nvml is not None:
+                    self._sample_nvml()
+                else:
+                    self._sample_smi()
             except Exception:
                 pass
-            self._stop.wait(0.1)
+            self._stop.wait(self.PERIOD_S)
 
     def __enter__(self):
         self._thread.start()
@@ -76,19 +130,9 @@ class ClockSampler:
         self._thread.join(timeout=10)
 
     def summary(self):
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for s in self.samples:
-            try:
-                sm.append(float(s[0]))
-                mx.append(float(s[1]))
-            except ValueError:
-                continue
-            for n, val in zip(names, s[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": max(self.mx) if self.mx else None,
+                "power_w_max": max(self.power) if self.power else None, "reasons": sorted(self.reasons),
+                "samples": len(self.sm), "source": self.source}
 
 
 def sample_rows_for_cpu(w, n_text_rows, n_img_rows, seed=0):
@@ -140,10 +184,26 @@ def time_oracle_sample(w, q, k, v, target_s=15.0):
                       f"{pairs} allowed pairs, {dt:.2f} s"}, dt, pairs
 
 
+def time_oracle_full(w, q, k, v):
+    """The oracle on the whole workload (every head, every row): for the workloads it finishes in seconds."""
+    from oracle import clear_oracle as oracle
+    pairs = int(allowed_counts(w).sum()) * w.B * w.H
+    t0 = time.perf_counter()
+    oracle.attn(q, k, v, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale)
+    dt = time.perf_counter() - t0
+    return {"value": 4.0 * pairs * w.head_dim / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"the whole workload ({pairs} allowed pairs), {dt:.2f} s"}
+
+
+FULL_ORACLE_WORKLOADS = ("c0_tiny_f32", "c1_1024px_r8", "c2_2048px_r16")
+
+
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
+    if args.steps is None:
+        args.steps = 5
     q, k, v = workloads.make_inputs(w, heads=1)
     per_step_target = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
     times, pairs_all = [], []
@@ -218,9 +278,17 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize()
 
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    plan.forward(qd, kd, vd, out, w.scale)
+    w0.record(stream)
     for _ in range(args.warmup):
         plan.forward(qd, kd, vd, out, w.scale)
+    w1.record(stream)
     plan.check()
+    if args.steps is None:
+        # no --steps given: as many as make the timed region last 0.6 s (same count on every rank)
+        warm_ms = max_over_ranks(w0.elapsed_time(w1) / args.warmup, dist, dev)
+        args.steps = int(min(2000, max(20, math.ceil(600.0 / max(warm_ms, 1e-3)))))
 
     # ---- device-resident timing -----------------------------------------------------------------
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
@@ -283,7 +351,9 @@ def run_ours(args, w):
             traffic = None
     if info.kernel != clear.KERNEL_SIMT:
         roofline = {"bound": "tensor", "achieved": per_gpu_tflops, "peak": peak, "unit": "TFLOP/s",
-                    "frac": per_gpu_tflops / peak, "traffic": traffic, "peak_kind": f"{peaks_kind} bf16 burst",
+                    "frac": per_gpu_tflops / peak, "traffic": traffic,
+                    "traffic_source": "stored ncu capture of this kernel (profiles/dram_traffic_per_launch.txt)"
+                    if traffic is not None else None, "peak_kind": f"{peaks_kind} bf16 burst",
                     "frac_of_sustained": per_gpu_tflops / float(peaks.get("bf16_tflops_sustained", peak)),
                     "executed_tflops": per_gpu_tflops * info.executed_pairs / info.sum_mask,
                     "geometric_efficiency": info.sum_mask / info.executed_pairs,
@@ -298,8 +368,13 @@ def run_ours(args, w):
 
     cpu_baseline = None
     if not args.no_cpu:
-        cpu_baseline, _, _ = time_oracle_sample(w, q[:, :1].contiguous(), k[:, :1].contiguous(),
-                                                v[:, :1].contiguous())
+        if w.name in FULL_ORACLE_WORKLOADS:
+            cpu_baseline = time_oracle_full(w, q, k, v)
+        else:
+            cpu_baseline, _, _ = time_oracle_sample(w, q[:, :1].contiguous(), k[:, :1].contiguous(),
+                                                    v[:, :1].contiguous())
+            cpu_baseline["sample"] += "; rate of the sample, the whole workload would take " \
+                                      f"{flops / (cpu_baseline['value'] * 1e12):.0f} s at it (extrapolated)"
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -307,6 +382,7 @@ def run_ours(args, w):
             "config": workload_config(w), "clocks": clock_info, "e2e": e2e,
             "gpu_launches": launches_per_call * args.steps, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "ms_min": float(min(ms)), "ms_median": float(np.median(ms)), "wall_s_timed_region": t_wall,
+            "ms_x_sm_mhz": ms_per_step * clock_info["sm_mhz"] if clock_info.get("sm_mhz") else None,
             "flops_per_call": flops, "sum_mask_per_head": info.sum_mask, "parallelism": "replicas"}
     print(json.dumps(line))
     if dist is not None:
@@ -317,8 +393,9 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default: as many as make the timed region last 0.6 s, at least 20)")
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="c4_8k_r16", choices=sorted(workloads.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
