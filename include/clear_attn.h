@@ -178,6 +178,13 @@ int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *
                        void *dv, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius,
                        float scale, void *stream);
 
+/* Window of an image query (text tokens are always allowed, as in Eq. 3). */
+enum {
+    CLEAR_MASK_DISC = 0,   /* Eq. 3: dx^2 + dy^2 < r^2, the paper's circular window                              */
+    CLEAR_MASK_SQUARE = 1  /* max(|dx|, |dy|) < r: the square sliding window of Neighborhood Attention, which
+                              Sec. 3.2 sets the circular one against (the circle costs about pi / 4 of it)      */
+};
+
 /* Build the schedule for one shape on the current device (Eq. 3 turned into integer geometry):
  * the threshold ceil(radius^2), for every 2-D query patch the list of key patches that meet its
  * radius-r dilation (with a flag telling whether the exact mask is needed) plus the text tiles,
@@ -187,6 +194,11 @@ int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *
  * Errors: INVALID_ARG, UNSUPPORTED (kernel/dtype/head_dim combination), CUDA, NO_MEMORY. */
 int clear_plan_create(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text,
                       int head_dim, float radius, int dtype, int kernel);
+
+/* clear_plan_create with the window kind chosen (CLEAR_MASK_*); every kernel serves both kinds, the schedule
+ * and its mask table are built for the window given.  Errors as clear_plan_create, INVALID_ARG for an unknown kind. */
+int clear_plan_create_ex(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text,
+                         int head_dim, float radius, int dtype, int kernel, int mask_kind, int host_only);
 
 /* The same schedule built on the host only: no CUDA call is made and no device is needed.  The
  * plan can be inspected (clear_plan_info, clear_plan_tables) and destroyed, not executed

@@ -18,6 +18,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_PLAN_MISMATCH = -1, -2, -3
 ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY, ERR_TOO_LARGE = -5, -6, -7, -8
 BF16, F32 = 0, 1
 KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_TCGEN05_WS = 0, 1, 2, 3
+MASK_DISC, MASK_SQUARE = 0, 1
 TILE_LINEAR, TILE_MASKED = 1, 2
 STEP_USE0, STEP_USE1, STEP_SHARED, STEP_LINEAR, STEP_MASKED0, STEP_MASKED1 = 1, 2, 4, 8, 16, 32
 STEP_CLIP0, STEP_CLIP1 = 64, 128
@@ -27,7 +28,7 @@ EXPORTS = [
     "clear_plan_tables", "clear_attn_fwd_planned", "clear_attn_fwd_host", "clear_plan_info",
     "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
     "clear_last_cuda_error", "clear_attn_fwd_static", "clear_plan_pair_tables",
-    "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim", "clear_attn_bwd_f32",
+    "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim", "clear_attn_bwd_f32", "clear_plan_create_ex",
 ]
 
 
@@ -94,6 +95,7 @@ def load() -> ctypes.CDLL:
         plan_args = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, f32, i32, i32]
         lib.clear_plan_create.argtypes = plan_args
         lib.clear_plan_create_host.argtypes = plan_args
+        lib.clear_plan_create_ex.argtypes = plan_args + [i32, i32]
         lib.clear_plan_tables.argtypes = [vp, ctypes.POINTER(ctypes.POINTER(WorkItem)), ctypes.POINTER(ctypes.c_int32),
                                           ctypes.POINTER(ctypes.POINTER(KvTile)), ctypes.POINTER(ctypes.c_int32),
                                           ctypes.POINTER(ctypes.POINTER(ctypes.c_int32)),
@@ -211,11 +213,16 @@ class Plan:
     """Owner of a ``clear_plan_t``."""
 
     def __init__(self, B, H, grid_h, grid_w, n_text, head_dim, radius, dtype=BF16, kernel=KERNEL_AUTO,
-                 host_only=False):
+                 host_only=False, mask_kind=MASK_DISC):
         self._h = ctypes.c_void_p()
-        fn = load().clear_plan_create_host if host_only else load().clear_plan_create
-        _check(fn(ctypes.byref(self._h), B, H, grid_h, grid_w, n_text, head_dim, float(radius), dtype, kernel),
-               "clear_plan_create_host" if host_only else "clear_plan_create")
+        if mask_kind != MASK_DISC:
+            _check(load().clear_plan_create_ex(ctypes.byref(self._h), B, H, grid_h, grid_w, n_text, head_dim,
+                                               float(radius), dtype, kernel, mask_kind, 1 if host_only else 0),
+                   "clear_plan_create_ex")
+        else:
+            fn = load().clear_plan_create_host if host_only else load().clear_plan_create
+            _check(fn(ctypes.byref(self._h), B, H, grid_h, grid_w, n_text, head_dim, float(radius), dtype, kernel),
+                   "clear_plan_create_host" if host_only else "clear_plan_create")
         self.dtype = dtype
 
     @property

@@ -369,6 +369,14 @@ int clear_plan_create(clear_plan_t **plan, int B, int H, int grid_h, int grid_w,
     return create_plan(plan, s, false);
 }
 
+int clear_plan_create_ex(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text, int head_dim,
+                         float radius, int dtype, int kernel, int mask_kind, int host_only)
+{
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, dtype, kernel};
+    s.mask_kind = mask_kind;
+    return create_plan(plan, s, host_only != 0);
+}
+
 int clear_plan_create_host(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text, int head_dim,
                            float radius, int dtype, int kernel)
 {

@@ -27,6 +27,7 @@ int validate_shape(const Shape &s)
     if (!(s.radius > 0.f) || !std::isfinite(s.radius)) return CLEAR_ERR_INVALID_ARG;
     if (s.dtype != CLEAR_BF16 && s.dtype != CLEAR_F32) return CLEAR_ERR_INVALID_ARG;
     if (s.kernel < CLEAR_KERNEL_AUTO || s.kernel > CLEAR_KERNEL_TCGEN05_WS) return CLEAR_ERR_INVALID_ARG;
+    if (s.mask_kind != CLEAR_MASK_DISC && s.mask_kind != CLEAR_MASK_SQUARE) return CLEAR_ERR_INVALID_ARG;
     const int64_t n = (int64_t)s.grid_h * s.grid_w;
     const int64_t N = n + s.n_text;
     if (N > (int64_t)1 << 30) return CLEAR_ERR_UNSUPPORTED;  // token indices stay in int32
@@ -53,11 +54,14 @@ void build_geometry(const Shape &s, Schedule &sch)
     const int64_t diag2 = (gh - 1) * (gh - 1) + (gw - 1) * (gw - 1);
     sch.thr = (r2 > (double)(diag2 + 1)) ? diag2 + 1 : (int64_t)r2;
 
-    const int64_t R = std::min<int64_t>(isqrt64(sch.thr - 1), gh - 1);  // largest |dy| that still has keys
+    // The window as half widths per row offset: the open disc of Eq. 3, or the square window of Neighborhood
+    // Attention (Sec. 3.2 sets the disc against it), max(|dx|, |dy|) < r, i.e. |dx|, |dy| <= ceil(r) - 1.
+    const int64_t reach = s.mask_kind == CLEAR_MASK_SQUARE ? (int64_t)std::ceil(r) - 1 : isqrt64(sch.thr - 1);
+    const int64_t R = std::min<int64_t>(reach, gh - 1);  // largest |dy| that still has keys
     sch.half_width.assign((size_t)R + 1, 0);
     int64_t img_img = 0;
     for (int64_t dy = 0; dy <= R; ++dy) {
-        const int64_t m = std::min<int64_t>(isqrt64(sch.thr - 1 - dy * dy), gw - 1);
+        const int64_t m = std::min<int64_t>(s.mask_kind == CLEAR_MASK_SQUARE ? reach : isqrt64(sch.thr - 1 - dy * dy), gw - 1);
         sch.half_width[(size_t)dy] = (int32_t)m;
         // keys in row y+dy seen by the gw queries of row y: sum_x (min(x+m, gw-1) - max(x-m, 0) + 1)
         const int64_t row_pairs = gw * (2 * m + 1) - m * (m + 1);
@@ -67,13 +71,22 @@ void build_geometry(const Shape &s, Schedule &sch)
     sch.sum_mask = T * N + n * T + img_img;
 }
 
+// The window of the schedule as a predicate on offsets: (dy, dx) is allowed iff |dx| <= half_width[|dy|].  The half
+// widths do not grow with |dy| (disc and square alike), so of two axis-aligned boxes of offsets SOME pair is allowed
+// iff the nearest one is, and EVERY pair iff the farthest one is.
+static bool window_allows(const Schedule &sch, int64_t dy, int64_t dx)
+{
+    dy = dy < 0 ? -dy : dy;
+    dx = dx < 0 ? -dx : dx;
+    return dy < (int64_t)sch.half_width.size() && dx <= sch.half_width[(size_t)dy];
+}
+
 void build_tile_schedule(const Shape &s, Schedule &sch)
 {
     build_geometry(s, sch);
     const int gh = s.grid_h, gw = s.grid_w, T = s.n_text;
     const int64_t N = (int64_t)gh * gw + T;
-    const int64_t thr = sch.thr;
-    const int R = (int)isqrt64(thr - 1);
+    const int R = (int)sch.half_width.size() - 1;  // rows a window reaches up and down
 
     sch.items.clear();
     sch.tiles.clear();
@@ -114,7 +127,7 @@ void build_tile_schedule(const Shape &s, Schedule &sch)
 
     // ---- image-query patches: text tiles, then the key patches that meet the dilated patch -----
     const int ntx = (gw + kTileW - 1) / kTileW, nty = (gh + kTileH - 1) / kTileH;
-    const int reach_x = R / kTileW + 1, reach_y = R / kTileH + 1;
+    const int reach_x = sch.half_width[0] / kTileW + 1, reach_y = R / kTileH + 1;
     for (int ty = 0; ty < nty; ++ty) {
         for (int tx = 0; tx < ntx; ++tx) {
             clear_work_item_t it{};
@@ -139,7 +152,7 @@ void build_tile_schedule(const Shape &s, Schedule &sch)
                     // smallest and largest coordinate differences between the two (clipped) patches
                     const int64_t gx = std::max({0, bx - qx1, it.qx - kx1});
                     const int64_t gy = std::max({0, by - qy1, it.qy - ky1});
-                    if (gx * gx + gy * gy >= thr) continue;
+                    if (!window_allows(sch, gy, gx)) continue;
                     const int64_t fx = std::max(kx1 - it.qx, qx1 - bx);
                     const int64_t fy = std::max(ky1 - it.qy, qy1 - by);
                     const bool whole = (bx + kTileW <= gw) && (by + kTileH <= gh);
@@ -147,7 +160,7 @@ void build_tile_schedule(const Shape &s, Schedule &sch)
                     kt.x = bx;
                     kt.y = by;
                     kt.n_valid = kTileTokens;
-                    kt.flags = (whole && fx * fx + fy * fy < thr) ? 0 : CLEAR_TILE_MASKED;
+                    kt.flags = (whole && window_allows(sch, fy, fx)) ? 0 : CLEAR_TILE_MASKED;
                     sch.tiles.push_back(kt);
                 }
             }
@@ -181,12 +194,12 @@ struct PatchTile {
 
 // Key patches (on the 8 x 16 lattice) that hold at least one key allowed to some query of the patch
 // at (qx, qy), each with the flag "some pair of the tile is not allowed".
-std::vector<PatchTile> patches_of(const Shape &s, int64_t thr, int R, int qx, int qy)
+std::vector<PatchTile> patches_of(const Shape &s, const Schedule &sch, int R, int qx, int qy)
 {
     const int gh = s.grid_h, gw = s.grid_w;
     const int ntx = (gw + kTileW - 1) / kTileW, nty = (gh + kTileH - 1) / kTileH;
     const int tx = qx / kTileW, ty = qy / kTileH;
-    const int reach_x = R / kTileW + 1, reach_y = R / kTileH + 1;
+    const int reach_x = sch.half_width[0] / kTileW + 1, reach_y = R / kTileH + 1;
     const int qx1 = std::min(qx + kTileW - 1, gw - 1), qy1 = std::min(qy + kTileH - 1, gh - 1);
     std::vector<PatchTile> out;
     for (int j = std::max(0, ty - reach_y); j <= std::min(nty - 1, ty + reach_y); ++j) {
@@ -195,11 +208,11 @@ std::vector<PatchTile> patches_of(const Shape &s, int64_t thr, int R, int qx, in
             const int kx1 = std::min(bx + kTileW - 1, gw - 1), ky1 = std::min(by + kTileH - 1, gh - 1);
             const int64_t gx = std::max({0, bx - qx1, qx - kx1});
             const int64_t gy = std::max({0, by - qy1, qy - ky1});
-            if (gx * gx + gy * gy >= thr) continue;
+            if (!window_allows(sch, gy, gx)) continue;
             const int64_t fx = std::max(kx1 - qx, qx1 - bx);
             const int64_t fy = std::max(ky1 - qy, qy1 - by);
             const bool whole = (bx + kTileW <= gw) && (by + kTileH <= gh);
-            out.push_back(PatchTile{bx, by, !(whole && fx * fx + fy * fy < thr), !whole});
+            out.push_back(PatchTile{bx, by, !(whole && window_allows(sch, fy, fx)), !whole});
         }
     }
     return out;
@@ -212,8 +225,7 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
     build_geometry(s, sch);
     const int gh = s.grid_h, gw = s.grid_w, T = s.n_text;
     const int64_t N = (int64_t)gh * gw + T;
-    const int64_t thr = sch.thr;
-    const int R = (int)isqrt64(thr - 1);
+    const int R = (int)sch.half_width.size() - 1;  // rows a window reaches up and down
 
     sch.pair_items.clear();
     sch.pair_steps.clear();
@@ -238,7 +250,7 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
             const int qy = r / kTileW, qx = r % kTileW;
             for (int j = 0; j < kTileTokens; ++j) {
                 const int64_t ddy = dy + j / kTileW - qy, ddx = dx + j % kTileW - qx;
-                if (ddx * ddx + ddy * ddy < thr) e[r * 4 + (j >> 5)] |= 1u << (j & 31);
+                if (window_allows(sch, ddy, ddx)) e[r * 4 + (j >> 5)] |= 1u << (j & 31);
             }
         }
         return id;
@@ -328,8 +340,8 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
             // text keys: tokens past n_text in the last tile are image keys, not allowed through it
             for (int t0 = 0; t0 < T; t0 += kTileTokens) linear_step(t0, std::min(kTileTokens, T - t0), it.n_sides);
 
-            std::vector<PatchTile> a = patches_of(s, thr, R, it.qx, it.qy0), b;
-            if (it.n_sides == 2) b = patches_of(s, thr, R, it.qx, it.qy1);
+            std::vector<PatchTile> a = patches_of(s, sch, R, it.qx, it.qy0), b;
+            if (it.n_sides == 2) b = patches_of(s, sch, R, it.qx, it.qy1);
             auto find = [](const std::vector<PatchTile> &v, const PatchTile &t) -> const PatchTile * {
                 for (const PatchTile &u : v)
                     if (u.x == t.x && u.y == t.y) return &u;

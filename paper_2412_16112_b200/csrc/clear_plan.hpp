@@ -19,16 +19,18 @@ struct Shape {
     float radius = 0.f;
     int dtype = 0;
     int kernel = 0;
+    int mask_kind = 0;  // CLEAR_MASK_DISC (Eq. 3) or CLEAR_MASK_SQUARE
     bool operator==(const Shape &o) const
     {
         return B == o.B && H == o.H && grid_h == o.grid_h && grid_w == o.grid_w && n_text == o.n_text &&
-               head_dim == o.head_dim && radius == o.radius && dtype == o.dtype && kernel == o.kernel;
+               head_dim == o.head_dim && radius == o.radius && dtype == o.dtype && kernel == o.kernel &&
+               mask_kind == o.mask_kind;
     }
 };
 
 struct Schedule {
-    int64_t thr = 0;                     // ceil(radius^2): allowed iff dx^2 + dy^2 < thr (Eq. 3)
-    std::vector<int32_t> half_width;     // half_width[dy] = max |dx| allowed at row offset dy
+    int64_t thr = 0;                     // ceil(radius^2): the disc allows dx^2 + dy^2 < thr (Eq. 3)
+    std::vector<int32_t> half_width;     // half_width[dy] = max |dx| allowed at row offset dy (the window, whatever its kind)
     std::vector<clear_work_item_t> items;
     std::vector<clear_kv_tile_t> tiles;
     std::vector<clear_pair_item_t> pair_items;   // TCGEN05_WS: text items first, then image items

@@ -578,3 +578,26 @@ def test_the_plan_cache_keeps_a_bounded_number_of_shapes(monkeypatch):
         assert_close_bf16(o.cpu(), oracle.attn(q, k, v, gh, 16, 5, 3.0, scale), f"cached shape {gh}")
     clear.clear_cache_clear()
     del outs
+
+
+# ----------------------------------------------------------------------------------------------
+# the square window through the same kernels
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("kernel", [clear.KERNEL_SIMT] + TC_KERNELS, ids=["simt"] + TC_IDS)
+@pytest.mark.parametrize("gh,gw,T,r", [(24, 40, 130, 8.0), (13, 19, 7, 2.5), (40, 24, 256, 16.0), (33, 50, 0, 5.0)])
+def test_square_window_matches_its_oracle(kernel, gh, gw, T, r):
+    from oracle import clear_oracle_windows as win
+    d = 128
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, seed=gh * 3 + gw)
+    scale = 1 / math.sqrt(d)
+    want = win.attn(q, k, v, gh, gw, T, win.SQUARE, r, 0, scale)
+    plan = clear.Plan(1, 2, gh, gw, T, d, r, kernel=kernel, mask_kind=clear.MASK_SQUARE)
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    out = torch.full_like(qd, float("nan"))
+    plan.forward(qd, kd, vd, out, scale)
+    plan.check()
+    assert_close_bf16(out.cpu(), want, f"square window r={r}")
+    # and it is not the disc: at these radii the corners of the square weigh in
+    disc = oracle.attn(q, k, v, gh, gw, T, r, scale)
+    assert np.abs(want - disc).max() > 1e-3
+    plan.destroy()

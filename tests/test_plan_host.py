@@ -398,3 +398,37 @@ def test_key_lists_beyond_the_step_records_positions_fall_back():
     assert p.info().kernel == clear.KERNEL_SIMT
     n = gh * gw
     assert p.info().sum_mask == n * n
+
+
+@pytest.mark.parametrize("gh,gw,T,r", [(16, 16, 16, 4.0), (13, 19, 7, 2.5), (40, 24, 256, 16.0), (4, 100, 3, 30.0)])
+def test_square_window_geometry_and_schedules(gh, gw, T, r):
+    """The square window of Neighborhood Attention through the same plan interface: half widths, sum(M) and the
+    mask table against the window oracle; every allowed pair lies in exactly one listed key tile."""
+    from oracle import clear_oracle_windows as win
+    total, _ = win.mask_counts(win.SQUARE, r, 0, gh, gw, T)
+    h = math.ceil(r) - 1
+    for kernel in (clear.KERNEL_SIMT, clear.KERNEL_TCGEN05, clear.KERNEL_TCGEN05_WS):
+        p = clear.Plan(1, 1, gh, gw, T, 128, r, kernel=kernel, host_only=True, mask_kind=clear.MASK_SQUARE)
+        assert p.info().sum_mask == total
+        _, _, hw = p.tables()
+        assert hw == [min(h, gw - 1)] * (min(h, gh - 1) + 1)
+    # tile kernel: the listed key tiles of every query patch hold every allowed key of its queries
+    p = clear.Plan(1, 1, gh, gw, T, 128, r, kernel=clear.KERNEL_TCGEN05, host_only=True, mask_kind=clear.MASK_SQUARE)
+    items, tiles, _ = p.tables()
+    N = T + gh * gw
+    for it in items:
+        if it.kind != 0:
+            continue
+        covered = np.zeros(N, dtype=bool)
+        for kt in tiles[it.tile_begin: it.tile_begin + it.tile_count]:
+            if kt.flags & clear.TILE_LINEAR:
+                covered[kt.x: kt.x + kt.n_valid] = True
+            else:
+                for yy in range(kt.y, min(kt.y + 8, gh)):
+                    covered[T + yy * gw + kt.x: T + yy * gw + min(kt.x + 16, gw)] = True
+        for qy in range(it.qy, min(it.qy + 8, gh)):
+            for qx in range(it.qx, min(it.qx + 16, gw)):
+                row = win.mask_row(win.SQUARE, r, 0, T + qy * gw + qx, gh, gw, T).astype(bool)
+                assert not (row & ~covered).any()
+    with pytest.raises(clear.ClearError):
+        clear.Plan(1, 1, gh, gw, T, 128, r, host_only=True, mask_kind=5)
