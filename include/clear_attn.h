@@ -178,6 +178,36 @@ int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *
                        void *dv, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius,
                        float scale, void *stream);
 
+/* What the model does to Q and K between their projections and the attention call, in one pass over memory:
+ * RMS normalisation over the head's channels, rotary position embedding on the two axes of the feature map
+ * (Sec. 3.1: the model perceives spatial relations through it, by the relative distances on the two axes), with
+ * the NTK factor on the rotary base that Sec. 4.3 raises from 1 to 10 beyond the training resolution, and a
+ * constant factor on Q (pass clear_log_scale_factor() for the log-scale attention factor of the same recipe, or
+ * leave it at 1 and multiply `scale` of the attention call instead).  For every (b, h) and token n with
+ * position (0, 0, 0) for text tokens and (0, y, x) for image token p = y * grid_w + x:
+ *     z   = x / sqrt(mean_c(x_c^2) + eps) * gain                                  (x = the row q[b,h,n,:] or k[b,h,n,:])
+ *     the head's channels form three groups of axis0_dim, axis1_dim, axis2_dim channels (in this order); in
+ *     group a of `dim` channels the pair (2j, 2j+1) turns by the angle position[a] * w_j,
+ *     w_j = base^(-2j/dim), base = theta * ntk_factor^(dim/(dim-2)) (base = theta when dim = 2):
+ *     out_2j = z_2j cos - z_2j+1 sin,   out_2j+1 = z_2j sin + z_2j+1 cos;   q_out is further multiplied by q_factor.
+ * q_in, k_in, q_out, k_out: device pointers, [B, H, N, head_dim] contiguous, N = n_text + grid_h * grid_w,
+ * bf16 (dtype CLEAR_BF16) or fp32 (CLEAR_F32), 16-byte aligned; arithmetic in fp32, frequencies from fp64 on
+ * the host; an output may be the very same pointer as its input (in place), any other overlap is not allowed.
+ * gain_q, gain_k: device pointers to head_dim fp32 values, or NULL for a gain of one.  The caller owns all
+ * buffers.  One kernel launch on `stream` (a cudaStream_t), no allocation, no host synchronisation.
+ * Errors: INVALID_ARG (sizes <= 0, n_text < 0, an odd or negative group size, groups not summing to head_dim,
+ * theta or ntk_factor <= 0 or non-finite, eps < 0, a non-finite value, a null tensor, unknown dtype),
+ * UNSUPPORTED (head_dim other than 64 or 128), MISALIGNED, CUDA. */
+int clear_qk_norm_rope(const void *q_in, const void *k_in, void *q_out, void *k_out, const float *gain_q,
+                       const float *gain_k, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, int dtype,
+                       int axis0_dim, int axis1_dim, int axis2_dim, float theta, float ntk_factor, float eps,
+                       float q_factor, void *stream);
+
+/* sqrt(log n_tokens / log n_train_tokens): the factor on the logits that keeps the entropy of the attention
+ * of a longer sequence where it was at the training length (the log-scale attention factor Sec. 4.3 applies
+ * beyond the training resolution).  Host arithmetic only; 1 when either count is below 2. */
+float clear_log_scale_factor(long long n_tokens, long long n_train_tokens);
+
 /* Window of an image query (text tokens are always allowed, as in Eq. 3). */
 enum {
     CLEAR_MASK_DISC = 0,   /* Eq. 3: dx^2 + dy^2 < r^2, the paper's circular window                              */

@@ -29,6 +29,7 @@ EXPORTS = [
     "clear_plan_check", "clear_plan_destroy", "clear_cache_clear", "clear_status_string",
     "clear_last_cuda_error", "clear_attn_fwd_static", "clear_plan_pair_tables",
     "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim", "clear_attn_bwd_f32", "clear_plan_create_ex",
+    "clear_qk_norm_rope", "clear_log_scale_factor",
 ]
 
 
@@ -92,6 +93,10 @@ def load() -> ctypes.CDLL:
         lib.clear_attn_fwd_f32.argtypes = fwd_args
         lib.clear_attn_fwd_static.argtypes = fwd_args
         lib.clear_attn_bwd_f32.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp]
+        lib.clear_qk_norm_rope.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, i32,
+                                           f32, f32, f32, f32, vp]
+        lib.clear_log_scale_factor.argtypes = [ctypes.c_longlong, ctypes.c_longlong]
+        lib.clear_log_scale_factor.restype = f32
         plan_args = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, f32, i32, i32]
         lib.clear_plan_create.argtypes = plan_args
         lib.clear_plan_create_host.argtypes = plan_args
@@ -119,7 +124,7 @@ def load() -> ctypes.CDLL:
         lib.clear_last_cuda_error.argtypes = []
         lib.clear_last_device_status.argtypes = []
         for name in EXPORTS:
-            if name != "clear_status_string":
+            if name not in ("clear_status_string", "clear_log_scale_factor"):
                 getattr(lib, name).restype = i32
         _lib = lib
         return lib
@@ -185,6 +190,34 @@ def clear_attn_bwd_f32(q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radiu
                                      dk.data_ptr(), dv.data_ptr(), B, H, grid_h, grid_w, n_text, d, float(radius),
                                      float(scale), _stream_ptr(stream)), "clear_attn_bwd_f32")
     return dq, dk, dv
+
+
+def clear_qk_norm_rope(q, k, q_out, k_out, grid_h, grid_w, n_text, axes_dim, gain_q=None, gain_k=None, theta=10000.0,
+                       ntk_factor=1.0, eps=1e-6, q_factor=1.0, stream=None):
+    """RMS normalisation, two-axis rotary embedding and the factor on Q, from ``q``, ``k`` into ``q_out``, ``k_out``
+    (bf16 or fp32 CUDA tensors of one [B, H, N, d] shape; an output may be its own input)."""
+    import torch
+    for t in (q, k, q_out, k_out):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == q.dtype and t.shape == q.shape):
+            raise ValueError("q, k and the outputs must be contiguous CUDA tensors of one dtype and [B, H, N, d] shape")
+    if q.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError("bf16 or fp32 tensors")
+    for g in (gain_q, gain_k):
+        if g is not None and not (g.is_cuda and g.is_contiguous() and g.dtype == torch.float32 and g.numel() == q.shape[-1]):
+            raise ValueError("a gain is a contiguous fp32 CUDA tensor of head_dim values")
+    B, H, _, d = q.shape
+    a0, a1, a2 = (int(a) for a in axes_dim)
+    _check(load().clear_qk_norm_rope(q.data_ptr(), k.data_ptr(), q_out.data_ptr(), k_out.data_ptr(),
+                                     gain_q.data_ptr() if gain_q is not None else None,
+                                     gain_k.data_ptr() if gain_k is not None else None,
+                                     B, H, grid_h, grid_w, n_text, d, BF16 if q.dtype == torch.bfloat16 else F32,
+                                     a0, a1, a2, float(theta), float(ntk_factor), float(eps), float(q_factor),
+                                     _stream_ptr(stream)), "clear_qk_norm_rope")
+    return q_out, k_out
+
+
+def clear_log_scale_factor(n_tokens: int, n_train_tokens: int) -> float:
+    return float(load().clear_log_scale_factor(int(n_tokens), int(n_train_tokens)))
 
 
 def clear_attn_fwd_f32(q, k, v, out, grid_h, grid_w, n_text, radius, scale, stream=None):

@@ -362,6 +362,34 @@ int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *
     });
 }
 
+int clear_qk_norm_rope(const void *q_in, const void *k_in, void *q_out, void *k_out, const float *gain_q,
+                       const float *gain_k, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, int dtype,
+                       int axis0_dim, int axis1_dim, int axis2_dim, float theta, float ntk_factor, float eps,
+                       float q_factor, void *stream)
+{
+    if (B <= 0 || H <= 0 || grid_h <= 0 || grid_w <= 0 || n_text < 0) return CLEAR_ERR_INVALID_ARG;
+    if (dtype != CLEAR_BF16 && dtype != CLEAR_F32) return CLEAR_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return CLEAR_ERR_UNSUPPORTED;
+    const int axes[3] = {axis0_dim, axis1_dim, axis2_dim};
+    for (int a = 0; a < 3; ++a)
+        if (axes[a] < 0 || (axes[a] & 1)) return CLEAR_ERR_INVALID_ARG;
+    if (axis0_dim + axis1_dim + axis2_dim != head_dim) return CLEAR_ERR_INVALID_ARG;
+    if (!(theta > 0.f) || !std::isfinite(theta) || !(ntk_factor > 0.f) || !std::isfinite(ntk_factor))
+        return CLEAR_ERR_INVALID_ARG;
+    if (!(eps >= 0.f) || !std::isfinite(eps) || !std::isfinite(q_factor)) return CLEAR_ERR_INVALID_ARG;
+    const int rc = check_tensors(q_in, k_in, q_out, k_out);
+    if (rc != CLEAR_OK) return rc;
+    if ((((uintptr_t)gain_q) | ((uintptr_t)gain_k)) & 3u) return CLEAR_ERR_MISALIGNED;
+    return launch_qk_prep(q_in, k_in, q_out, k_out, gain_q, gain_k, B * H, grid_h, grid_w, n_text, head_dim, dtype, axes,
+                          (double)theta, (double)ntk_factor, eps, q_factor, static_cast<cudaStream_t>(stream));
+}
+
+float clear_log_scale_factor(long long n_tokens, long long n_train_tokens)
+{
+    if (n_tokens < 2 || n_train_tokens < 2) return 1.f;
+    return (float)std::sqrt(std::log((double)n_tokens) / std::log((double)n_train_tokens));
+}
+
 int clear_plan_create(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text, int head_dim,
                       float radius, int dtype, int kernel)
 {

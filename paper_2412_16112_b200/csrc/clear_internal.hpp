@@ -100,6 +100,10 @@ int launch_ws(const clear_plan &p, const void *q, const void *k, const void *v, 
 // fp32 backward pass on the CUDA cores (dk and dv are zeroed on the stream first).
 int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq,
                    void *dk, void *dv, float scale, cudaStream_t stream);
+// Q/K preparation (RMS normalisation, rotary embedding, factor on Q): one elementwise pass, no plan.
+int launch_qk_prep(const void *q_in, const void *k_in, void *q_out, void *k_out, const float *gain_q, const float *gain_k,
+                   int n_bh, int grid_h, int grid_w, int n_text, int head_dim, int dtype, const int axes_dim[3],
+                   double theta, double ntk_factor, float eps, float q_factor, cudaStream_t stream);
 // Merge of the split-KV partial results of the text-query rows (both tensor-core kernels).
 int launch_text_combine(const clear_plan &p, void *out, cudaStream_t stream);
 

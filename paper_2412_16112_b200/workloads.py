@@ -93,3 +93,12 @@ def make_custom(B, H, grid_h, grid_w, n_text, head_dim, dtype="bf16", qk_norm=Tr
     """Inputs for an ad-hoc shape with the same value distribution."""
     w = Workload("custom", B, H, head_dim, grid_h, grid_w, n_text, 1.0, dtype, qk_norm, seed)
     return make_inputs(w)
+
+
+def make_gains(head_dim: int, seed: int = 0) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Gain vectors of a Q and a K normalisation layer, fp32 [head_dim]: 1 + 0.1 N(0, 1) (learned gains stay
+    near their initial value of one)."""
+    gen = torch.Generator(device="cpu").manual_seed(7000 + seed)
+    gq = 1.0 + 0.1 * torch.randn(head_dim, generator=gen, dtype=torch.float32)
+    gk = 1.0 + 0.1 * torch.randn(head_dim, generator=gen, dtype=torch.float32)
+    return gq, gk
