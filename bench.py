@@ -7,6 +7,8 @@ Prints ONE JSON line.  `value` is effective TFLOP/s, 4 * sum(M) * head_dim * H *
 4 * sum(M) * c), with q, k, v resident in HBM; `e2e` is the same metric through the host-tensor C-ABI
 entry point with the host<->device copies inside the timed region.  With N > 1 (torchrun) every rank runs
 an independent replica of the workload on its own GPU: the path has no exchange step.
+`qk_prep` times, outside `value`, the one-pass Q/K preparation kernel (normalisation + rotary embedding) on the
+same shape against the HBM copy rate.
 `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload (rank 0 only).
 """
 from __future__ import annotations
@@ -366,6 +368,30 @@ def run_ours(args, w):
                     "frac": per_gpu_tflops / alu_peak, "traffic": traffic, "peak_kind": "148 SMs x 128 fp32 FMA lanes",
                     "kernel": "clear_simt_kernel"}
 
+    # ---- the Q/K preparation that precedes the attention call in the model (outside `value`) -------------
+    qk_prep = None
+    if not args.no_prep and w.head_dim in (64, 128):
+        axes = (16, 56, 56) if w.head_dim == 128 else (8, 28, 28)
+        k_out = torch.empty_like(kd)
+        n_prep = 20
+        for _ in range(3):
+            clear.clear_qk_norm_rope(qd, kd, out, k_out, w.grid_h, w.grid_w, w.n_text, axes, ntk_factor=10.0)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        p0.record(stream)
+        for _ in range(n_prep):
+            clear.clear_qk_norm_rope(qd, kd, out, k_out, w.grid_h, w.grid_w, w.n_text, axes, ntk_factor=10.0)
+        p1.record(stream)
+        torch.cuda.synchronize()
+        prep_ms = p0.elapsed_time(p1) / n_prep
+        prep_bytes = 4 * qd.numel() * qd.element_size()   # Q and K read once and written once
+        hbm_peak = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+        qk_prep = {"kernel": "clear_qk_prep_kernel", "ms": prep_ms, "bound": "hbm", "achieved": prep_bytes / prep_ms / 1e6,
+                   "peak": hbm_peak, "unit": "GB/s", "frac": prep_bytes / prep_ms / 1e6 / hbm_peak,
+                   "peak_kind": f"{peaks_kind} copy", "bytes_per_launch": prep_bytes, "launches": n_prep,
+                   "note": "tensors fit in L2: no HBM figure" if small else "tensors larger than L2"}
+        del k_out
+
     cpu_baseline = None
     if not args.no_cpu:
         if w.name in FULL_ORACLE_WORKLOADS:
@@ -383,7 +409,8 @@ def run_ours(args, w):
             "gpu_launches": launches_per_call * args.steps, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "ms_min": float(min(ms)), "ms_median": float(np.median(ms)), "wall_s_timed_region": t_wall,
             "ms_x_sm_mhz": ms_per_step * clock_info["sm_mhz"] if clock_info.get("sm_mhz") else None,
-            "flops_per_call": flops, "sum_mask_per_head": info.sum_mask, "parallelism": "replicas"}
+            "flops_per_call": flops, "sum_mask_per_head": info.sum_mask, "parallelism": "replicas",
+            "qk_prep": qk_prep}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -399,6 +426,7 @@ def main():
     ap.add_argument("--workload", default="c4_8k_r16", choices=sorted(workloads.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-prep", action="store_true", help="skip the timing of the Q/K preparation kernel")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

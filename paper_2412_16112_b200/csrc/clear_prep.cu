@@ -4,9 +4,10 @@
 //
 // The work is elementwise with one reduction per row of d channels, so HBM bounds it: every element of Q and
 // K is read once and written once (4 * B * H * N * d * sizeof(element) bytes per call).  One warp owns one
-// token position and walks over all (batch, head) rows of that token: the angles depend on the position
-// only, so their sines and cosines are computed once per token and reused for 2 * B * H rows; a lane holds
-// d / 32 consecutive channels of a row (whole rotary pairs), so a row is one coalesced d-element access.
+// few token positions (32 / (d / 8) of them) and walks over all (batch, head) rows of those tokens: the angles
+// depend on the position only, so their sines and cosines are computed once per token and reused for
+// 2 * B * H rows; a lane holds 8 consecutive channels of a row (whole rotary pairs), so a row is one
+// coalesced access of 16 bytes per lane for bf16.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -33,104 +34,97 @@ struct PrepParams {
     uint8_t axis[kMaxPairs];       // which coordinate of the token's position turns pair p: 0 none, 1 y, 2 x
 };
 
-template <typename T, int EPL> struct RowIo;
-template <> struct RowIo<__nv_bfloat16, 4> {
-    static __device__ __forceinline__ void load(const void *base, long long elem, float (&x)[4])
+// Eight consecutive channels of a row (four rotary pairs) per lane: one 16-byte access for bf16, two for fp32.
+template <typename T> struct RowIo;
+template <> struct RowIo<__nv_bfloat16> {
+    static __device__ __forceinline__ void load(const void *base, long long elem, float (&x)[8])
     {
-        const uint2 u = *reinterpret_cast<const uint2 *>(static_cast<const __nv_bfloat16 *>(base) + elem);
-        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u.x));
-        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u.y));
-        x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+        const uint4 u = *reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(base) + elem);
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);            // a bf16 is the upper half of an fp32
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
     }
-    static __device__ __forceinline__ void store(void *base, long long elem, const float (&x)[4])
+    static __device__ __forceinline__ void store(void *base, long long elem, const float (&x)[8])
     {
-        uint2 u;
-        *reinterpret_cast<__nv_bfloat162 *>(&u.x) = __floats2bfloat162_rn(x[0], x[1]);
-        *reinterpret_cast<__nv_bfloat162 *>(&u.y) = __floats2bfloat162_rn(x[2], x[3]);
-        *reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(base) + elem) = u;
-    }
-};
-template <> struct RowIo<__nv_bfloat16, 2> {
-    static __device__ __forceinline__ void load(const void *base, long long elem, float (&x)[2])
-    {
-        const uint32_t u = *reinterpret_cast<const uint32_t *>(static_cast<const __nv_bfloat16 *>(base) + elem);
-        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u));
-        x[0] = a.x; x[1] = a.y;
-    }
-    static __device__ __forceinline__ void store(void *base, long long elem, const float (&x)[2])
-    {
-        uint32_t u;
-        *reinterpret_cast<__nv_bfloat162 *>(&u) = __floats2bfloat162_rn(x[0], x[1]);
-        *reinterpret_cast<uint32_t *>(static_cast<__nv_bfloat16 *>(base) + elem) = u;
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) *reinterpret_cast<__nv_bfloat162 *>(&w[i]) = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+        *reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(base) + elem) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 };
-template <> struct RowIo<float, 4> {
-    static __device__ __forceinline__ void load(const void *base, long long elem, float (&x)[4])
+template <> struct RowIo<float> {
+    static __device__ __forceinline__ void load(const void *base, long long elem, float (&x)[8])
     {
-        const float4 v = *reinterpret_cast<const float4 *>(static_cast<const float *>(base) + elem);
-        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+        const float4 a = *reinterpret_cast<const float4 *>(static_cast<const float *>(base) + elem);
+        const float4 b = *reinterpret_cast<const float4 *>(static_cast<const float *>(base) + elem + 4);
+        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+        x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
     }
-    static __device__ __forceinline__ void store(void *base, long long elem, const float (&x)[4])
+    static __device__ __forceinline__ void store(void *base, long long elem, const float (&x)[8])
     {
         *reinterpret_cast<float4 *>(static_cast<float *>(base) + elem) = make_float4(x[0], x[1], x[2], x[3]);
-    }
-};
-template <> struct RowIo<float, 2> {
-    static __device__ __forceinline__ void load(const void *base, long long elem, float (&x)[2])
-    {
-        const float2 v = *reinterpret_cast<const float2 *>(static_cast<const float *>(base) + elem);
-        x[0] = v.x; x[1] = v.y;
-    }
-    static __device__ __forceinline__ void store(void *base, long long elem, const float (&x)[2])
-    {
-        *reinterpret_cast<float2 *>(static_cast<float *>(base) + elem) = make_float2(x[0], x[1]);
+        *reinterpret_cast<float4 *>(static_cast<float *>(base) + elem + 4) = make_float4(x[4], x[5], x[6], x[7]);
     }
 };
 
-// One row: x -> x / sqrt(mean(x^2) + eps) * gain, every pair turned by its angle, times `factor`.
-template <int EPL, int D>
-__device__ __forceinline__ void prep_row(float (&x)[EPL], const float (&g)[EPL], const float (&cs)[EPL / 2][2], float eps,
-                                         float factor)
+constexpr int kEpl = 8;  // channels per lane
+
+// One row: x -> x / sqrt(mean(x^2) + eps) * gain, every pair turned by its angle, times `factor`.  The lanes
+// that share the row exchange their partial sums of squares; `gcs` holds, per pair, the products of the two
+// channels' gains with the pair's cosine and sine (they do not change from row to row of a token).
+template <int D>
+__device__ __forceinline__ void prep_row(float (&x)[kEpl], const float (&gcs)[kEpl / 2][4], float eps, float factor)
 {
     float ss = 0.f;
 #pragma unroll
-    for (int i = 0; i < EPL; ++i) ss = fmaf(x[i], x[i], ss);
+    for (int i = 0; i < kEpl; ++i) ss = fmaf(x[i], x[i], ss);
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-    const float inv = factor / sqrtf(ss * (1.f / D) + eps);
+    for (int off = D / kEpl / 2; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+    const float inv = factor * rsqrtf(fmaf(ss, 1.f / D, eps));
 #pragma unroll
-    for (int p = 0; p < EPL / 2; ++p) {
-        const float a = x[2 * p] * g[2 * p] * inv, b = x[2 * p + 1] * g[2 * p + 1] * inv;
-        x[2 * p] = a * cs[p][0] - b * cs[p][1];
-        x[2 * p + 1] = a * cs[p][1] + b * cs[p][0];
+    for (int p = 0; p < kEpl / 2; ++p) {
+        const float a = x[2 * p], b = x[2 * p + 1];
+        x[2 * p] = (a * gcs[p][0] - b * gcs[p][1]) * inv;      // g_a a cos - g_b b sin
+        x[2 * p + 1] = (a * gcs[p][2] + b * gcs[p][3]) * inv;  // g_a a sin + g_b b cos
     }
 }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kPrepThreads, 3) clear_qk_prep_kernel(const __grid_constant__ PrepParams prm)
+__global__ void __launch_bounds__(kPrepThreads, 2) clear_qk_prep_kernel(const __grid_constant__ PrepParams prm)
 {
-    constexpr int EPL = D / 32;  // channels per lane
-    constexpr int kRows = 4;     // rows in flight per lane and tensor
-    using Io = RowIo<T, EPL>;
+    constexpr int kLanesPerRow = D / kEpl;           // 16 or 8 lanes share a row
+    constexpr int kTokensPerWarp = 32 / kLanesPerRow;
+    constexpr int kRows = 4;                         // rows in flight per lane and tensor
+    using Io = RowIo<T>;
     const int lane = threadIdx.x & 31;
-    const long long warp0 = (long long)blockIdx.x * kPrepWarps + (threadIdx.x >> 5);
-    const long long n_warps = (long long)gridDim.x * kPrepWarps;
-    const int c0 = lane * EPL;
+    const int sub = lane / kLanesPerRow;             // which of the warp's tokens
+    const int c0 = (lane % kLanesPerRow) * kEpl;
+    const long long group0 = (long long)blockIdx.x * kPrepWarps + (threadIdx.x >> 5);
+    const long long n_groups = (long long)gridDim.x * kPrepWarps;
 
-    float gq[EPL], gk[EPL], freq[EPL / 2];
-    int axis[EPL / 2];
+    float gq[kEpl], gk[kEpl], freq[kEpl / 2];
+    int axis[kEpl / 2];
 #pragma unroll
-    for (int i = 0; i < EPL; ++i) {
+    for (int i = 0; i < kEpl; ++i) {
         gq[i] = prm.gain_q ? __ldg(prm.gain_q + c0 + i) : 1.f;
         gk[i] = prm.gain_k ? __ldg(prm.gain_k + c0 + i) : 1.f;
     }
 #pragma unroll
-    for (int p = 0; p < EPL / 2; ++p) {
+    for (int p = 0; p < kEpl / 2; ++p) {
         freq[p] = prm.freq[c0 / 2 + p];
         axis[p] = prm.axis[c0 / 2 + p];
     }
 
-    for (long long n = warp0; n < prm.n_tokens; n += n_warps) {
+    const long long row_stride = prm.n_tokens * D;
+    for (long long grp = group0; grp * kTokensPerWarp < prm.n_tokens; grp += n_groups) {
+        // the lanes of a token beyond the last one follow the last token and store nothing (the row's lanes
+        // stay together for the shuffles)
+        const long long n_raw = grp * kTokensPerWarp + sub;
+        const bool live = n_raw < prm.n_tokens;
+        const long long n = live ? n_raw : prm.n_tokens - 1;
         // position of the token: text tokens at the origin, image token p at (y, x) = (p / grid_w, p % grid_w)
         int pos_y = 0, pos_x = 0;
         if (n >= prm.n_text) {
@@ -138,17 +132,21 @@ __global__ void __launch_bounds__(kPrepThreads, 3) clear_qk_prep_kernel(const __
             pos_y = (int)(p / prm.grid_w);
             pos_x = (int)(p - (long long)pos_y * prm.grid_w);
         }
-        float cs[EPL / 2][2];
+        float gcs_q[kEpl / 2][4], gcs_k[kEpl / 2][4];
 #pragma unroll
-        for (int p = 0; p < EPL / 2; ++p) {
+        for (int p = 0; p < kEpl / 2; ++p) {
             const int pos = axis[p] == 1 ? pos_y : (axis[p] == 2 ? pos_x : 0);
-            sincosf((float)pos * freq[p], &cs[p][1], &cs[p][0]);
+            float sn, cs;
+            sincosf((float)pos * freq[p], &sn, &cs);
+            gcs_q[p][0] = gq[2 * p] * cs; gcs_q[p][1] = gq[2 * p + 1] * sn;
+            gcs_q[p][2] = gq[2 * p] * sn; gcs_q[p][3] = gq[2 * p + 1] * cs;
+            gcs_k[p][0] = gk[2 * p] * cs; gcs_k[p][1] = gk[2 * p + 1] * sn;
+            gcs_k[p][2] = gk[2 * p] * sn; gcs_k[p][3] = gk[2 * p + 1] * cs;
         }
         long long elem = n * D + c0;
-        const long long row_stride = prm.n_tokens * D;
         int bh = 0;
         for (; bh + kRows <= prm.n_bh; bh += kRows) {
-            float xq[kRows][EPL], xk[kRows][EPL];
+            float xq[kRows][kEpl], xk[kRows][kEpl];
 #pragma unroll
             for (int j = 0; j < kRows; ++j) {
                 Io::load(prm.q_in, elem + j * row_stride, xq[j]);
@@ -156,21 +154,25 @@ __global__ void __launch_bounds__(kPrepThreads, 3) clear_qk_prep_kernel(const __
             }
 #pragma unroll
             for (int j = 0; j < kRows; ++j) {
-                prep_row<EPL, D>(xq[j], gq, cs, prm.eps, prm.q_factor);
-                prep_row<EPL, D>(xk[j], gk, cs, prm.eps, 1.f);
-                Io::store(prm.q_out, elem + j * row_stride, xq[j]);
-                Io::store(prm.k_out, elem + j * row_stride, xk[j]);
+                prep_row<D>(xq[j], gcs_q, prm.eps, prm.q_factor);
+                prep_row<D>(xk[j], gcs_k, prm.eps, 1.f);
+                if (live) {
+                    Io::store(prm.q_out, elem + j * row_stride, xq[j]);
+                    Io::store(prm.k_out, elem + j * row_stride, xk[j]);
+                }
             }
             elem += kRows * row_stride;
         }
         for (; bh < prm.n_bh; ++bh) {
-            float xq[EPL], xk[EPL];
+            float xq[kEpl], xk[kEpl];
             Io::load(prm.q_in, elem, xq);
             Io::load(prm.k_in, elem, xk);
-            prep_row<EPL, D>(xq, gq, cs, prm.eps, prm.q_factor);
-            prep_row<EPL, D>(xk, gk, cs, prm.eps, 1.f);
-            Io::store(prm.q_out, elem, xq);
-            Io::store(prm.k_out, elem, xk);
+            prep_row<D>(xq, gcs_q, prm.eps, prm.q_factor);
+            prep_row<D>(xk, gcs_k, prm.eps, 1.f);
+            if (live) {
+                Io::store(prm.q_out, elem, xq);
+                Io::store(prm.k_out, elem, xk);
+            }
             elem += row_stride;
         }
     }
@@ -215,7 +217,8 @@ int launch_qk_prep(const void *q_in, const void *k_in, void *q_out, void *k_out,
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kPrepThreads, 0) != cudaSuccess || per_sm < 1)
             return CLEAR_ERR_CUDA;
         long long blocks = (long long)n_sm * per_sm;
-        const long long need = (prm.n_tokens + kPrepWarps - 1) / kPrepWarps;
+        const long long tokens_per_block = (long long)kPrepWarps * (32 / (head_dim / kEpl));
+        const long long need = (prm.n_tokens + tokens_per_block - 1) / tokens_per_block;
         if (blocks > need) blocks = need;
         kernel<<<dim3((unsigned)blocks), dim3(kPrepThreads), 0, stream>>>(prm);
         return CLEAR_OK;
