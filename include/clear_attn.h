@@ -230,6 +230,71 @@ int clear_plan_create(clear_plan_t **plan, int B, int H, int grid_h, int grid_w,
 int clear_plan_create_ex(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text,
                          int head_dim, float radius, int dtype, int kernel, int mask_kind, int host_only);
 
+/* ---- Row-band parallel form (Sec. 3.4) --------------------------------------------------------------------
+ * The H x W feature map is cut into bands of rows, one per GPU; every GPU also holds the text tokens.  An image
+ * query sees keys at most `reach` rows away (Eq. 3), so a GPU needs, besides its band, `halo_lo` rows above and
+ * `halo_hi` rows below it, which its neighbours send ("communication only in the boundary areas").  A GPU's LOCAL
+ * tensors are [B, H, n_text + local_rows * grid_w, head_dim] with local_rows = halo_lo + (y1 - y0) + halo_hi: the
+ * text tokens, then the rows y0 - halo_lo .. y1 + halo_hi - 1 of the grid, row-major; the band sits at local rows
+ * [halo_lo, halo_lo + y1 - y0).  Q and the output need only hold valid data in the text and band rows.
+ *   image queries of the band: a CLEAR_PART_BAND_IMAGE plan over the local grid, run by clear_attn_fwd_planned:
+ *       exactly the rows of the single-GPU result (the halo holds every key such a query can see, and the local
+ *       grid's border is the true border wherever a window reaches it);
+ *   text queries: they see every key, so each GPU computes them over ITS keys only -- a CLEAR_PART_BAND_TEXT plan,
+ *       run by clear_attn_text_partial, leaves per text row the un-normalised output with the row's maximum and
+ *       sum -- and clear_text_merge combines the records of all GPUs: exactly (the merge of a split softmax, Eq. 1
+ *       unchanged), or by the patch-wise average of Eq. 7.  Either way one record of head_dim + 2 floats per
+ *       text row and (b, h) is all that travels.
+ * The exchange itself (halo rows to the neighbours, records to everyone) is the caller's: the Python package does
+ * it with torch.distributed send/recv and all-gather into local buffers. */
+enum {
+    CLEAR_PART_ALL = 0,         /* an ordinary plan: the whole operator on one GPU                                  */
+    CLEAR_PART_BAND_IMAGE = 1,  /* the image queries of the band's rows                                             */
+    CLEAR_PART_BAND_TEXT = 2    /* the text queries over this GPU's keys, as records for clear_text_merge          */
+};
+enum {
+    CLEAR_TEXT_MERGE_EXACT = 0,   /* sum_p w_p O_p / sum_p w_p l_p, w_p = 2^(m_p - max m): the exact text rows       */
+    CLEAR_TEXT_MERGE_AVERAGE = 1  /* Eq. 7: (1 / n_parts) sum_p O_p / l_p                                            */
+};
+
+/* Rows [*y0, *y1) of band `band` when grid_h rows are cut into n_bands bands as evenly as possible (the first
+ * grid_h % n_bands bands are one row taller), and the halo rows the band needs above and below: the window's
+ * reach (largest |dy| with a visible key: dy^2 < ceil(radius^2) for the disc, ceil(radius) - 1 for the square),
+ * clipped at the grid's border.  Host arithmetic only; any output pointer may be NULL.
+ * Errors: INVALID_ARG (n_bands < 1 or > grid_h, band out of range, radius <= 0 or non-finite, unknown kind). */
+int clear_band_geometry(int grid_h, float radius, int mask_kind, int n_bands, int band, int32_t *y0, int32_t *y1,
+                        int32_t *halo_lo, int32_t *halo_hi);
+
+/* Plan of one part of a band (bf16, head_dim 64 or 128, the warp-specialised tensor-core kernel) over the LOCAL
+ * grid of local_rows x grid_w; the band is local rows [q_row_begin, q_row_end).
+ *   CLEAR_PART_BAND_IMAGE: work items for the 8 x 16 query patches that hold rows of the band.  Output rows of those
+ *       patches that lie outside the band are written too (with values the caller must ignore); text rows and all
+ *       other rows of `out` are left alone.
+ *   CLEAR_PART_BAND_TEXT: work items for the text queries over the image tokens of the band's own rows, and over
+ *       the text tokens too iff text_keys != 0.  For the exact merge exactly one GPU counts the text keys
+ *       (text_keys = 1 on band 0, 0 elsewhere); for Eq. 7 every GPU does.  Needs n_text > 0.
+ * clear_plan_info reports the allowed pairs and flops of the part.  Ownership, host_only and errors as
+ * clear_plan_create_ex; INVALID_ARG also for an empty or out-of-range band, an unknown part. */
+int clear_plan_create_band(clear_plan_t **plan, int B, int H, int local_rows, int grid_w, int n_text, int head_dim,
+                           float radius, int mask_kind, int part, int q_row_begin, int q_row_end, int text_keys,
+                           int host_only);
+
+/* Text queries over this GPU's keys (a CLEAR_PART_BAND_TEXT plan; q, k, v local tensors as above).  `records`:
+ * device pointer, [B * H][n_text][head_dim + 2] fp32, 16-byte aligned, fully written: head_dim values of
+ * sum_j 2^(s_ij - m_i) v_j over the keys j this GPU counts (s = scale * log2(e) * q_i . k_j), then m_i, then
+ * l_i = sum_j 2^(s_ij - m_i).  Streams, ordering and errors as clear_attn_fwd_planned; PLAN_MISMATCH for any
+ * other kind of plan (and clear_attn_fwd_planned returns PLAN_MISMATCH for this kind). */
+int clear_attn_text_partial(const clear_plan_t *plan, const void *q, const void *k, const void *v, float *records,
+                            float scale, void *stream);
+
+/* Merge of the records of all bands into the text rows: `records` is [n_parts][B * H][n_text][head_dim + 2] fp32
+ * on the device (the parts' records one after the other, e.g. as an all-gather leaves them), `out` a bf16
+ * [B, H, out_tokens, head_dim] tensor whose first n_text rows per (b, h) are written (16-byte aligned).  mode:
+ * CLEAR_TEXT_MERGE_EXACT or CLEAR_TEXT_MERGE_AVERAGE (Eq. 7).  One small kernel on `stream`, no allocation.
+ * Errors: INVALID_ARG, UNSUPPORTED (head_dim other than 64 or 128, B * H > 65535), MISALIGNED, CUDA. */
+int clear_text_merge(const float *records, int n_parts, int B, int H, int n_text, int head_dim, int mode, void *out,
+                     long long out_tokens, void *stream);
+
 /* The same schedule built on the host only: no CUDA call is made and no device is needed.  The
  * plan can be inspected (clear_plan_info, clear_plan_tables) and destroyed, not executed
  * (forward calls return PLAN_MISMATCH).  Errors: INVALID_ARG, UNSUPPORTED, NO_MEMORY. */

@@ -19,6 +19,8 @@ ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY, ERR_TOO_LARGE = -5, -6, -7, -8
 BF16, F32 = 0, 1
 KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_TCGEN05_WS = 0, 1, 2, 3
 MASK_DISC, MASK_SQUARE = 0, 1
+PART_ALL, PART_BAND_IMAGE, PART_BAND_TEXT = 0, 1, 2
+TEXT_MERGE_EXACT, TEXT_MERGE_AVERAGE = 0, 1
 TILE_LINEAR, TILE_MASKED = 1, 2
 STEP_USE0, STEP_USE1, STEP_SHARED, STEP_LINEAR, STEP_MASKED0, STEP_MASKED1 = 1, 2, 4, 8, 16, 32
 STEP_CLIP0, STEP_CLIP1 = 64, 128
@@ -30,6 +32,7 @@ EXPORTS = [
     "clear_last_cuda_error", "clear_attn_fwd_static", "clear_plan_pair_tables",
     "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim", "clear_attn_bwd_f32", "clear_plan_create_ex",
     "clear_qk_norm_rope", "clear_log_scale_factor",
+    "clear_band_geometry", "clear_plan_create_band", "clear_attn_text_partial", "clear_text_merge",
 ]
 
 
@@ -95,6 +98,12 @@ def load() -> ctypes.CDLL:
         lib.clear_attn_bwd_f32.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp]
         lib.clear_qk_norm_rope.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, i32,
                                            f32, f32, f32, f32, vp]
+        pi32 = ctypes.POINTER(ctypes.c_int32)
+        lib.clear_band_geometry.argtypes = [i32, f32, i32, i32, i32, pi32, pi32, pi32, pi32]
+        lib.clear_plan_create_band.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, f32, i32, i32, i32, i32,
+                                               i32, i32]
+        lib.clear_attn_text_partial.argtypes = [vp, vp, vp, vp, vp, f32, vp]
+        lib.clear_text_merge.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, ctypes.c_longlong, vp]
         lib.clear_log_scale_factor.argtypes = [ctypes.c_longlong, ctypes.c_longlong]
         lib.clear_log_scale_factor.restype = f32
         plan_args = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, f32, i32, i32]
@@ -324,6 +333,52 @@ class Plan:
             self.destroy()
         except Exception:
             pass
+
+
+class BandPlan(Plan):
+    """Plan of one part (``PART_BAND_IMAGE`` or ``PART_BAND_TEXT``) of a row band over its local grid."""
+
+    def __init__(self, B, H, local_rows, grid_w, n_text, head_dim, radius, part, q_row_begin, q_row_end,
+                 text_keys=True, mask_kind=MASK_DISC, host_only=False):
+        self._h = ctypes.c_void_p()
+        _check(load().clear_plan_create_band(ctypes.byref(self._h), B, H, local_rows, grid_w, n_text, head_dim,
+                                             float(radius), mask_kind, part, q_row_begin, q_row_end,
+                                             1 if text_keys else 0, 1 if host_only else 0), "clear_plan_create_band")
+        self.dtype = BF16
+        self.part = part
+
+    def text_partial(self, q, k, v, records, scale, stream=None):
+        """Records [B * H, n_text, d + 2] (fp32) of the text queries over this band's keys."""
+        import torch
+        ptrs = _tensor_args(q, k, v, q, BF16)
+        if not (records.is_cuda and records.is_contiguous() and records.dtype == torch.float32):
+            raise ValueError("records must be a contiguous fp32 CUDA tensor")
+        _check(load().clear_attn_text_partial(self._h, ptrs[0], ptrs[1], ptrs[2], records.data_ptr(), float(scale),
+                                              _stream_ptr(stream)), "clear_attn_text_partial")
+        return records
+
+
+def band_geometry(grid_h, radius, n_bands, band, mask_kind=MASK_DISC):
+    """(y0, y1, halo_lo, halo_hi) of one band."""
+    vals = [ctypes.c_int32() for _ in range(4)]
+    _check(load().clear_band_geometry(grid_h, float(radius), mask_kind, n_bands, band, *[ctypes.byref(x) for x in vals]),
+           "clear_band_geometry")
+    return tuple(x.value for x in vals)
+
+
+def clear_text_merge(records, out, n_text, mode=TEXT_MERGE_EXACT, stream=None):
+    """Merge the bands' records [n_parts, B * H, n_text, d + 2] into the first n_text rows of ``out`` [B, H, N, d]."""
+    import torch
+    if not (records.is_cuda and records.is_contiguous() and records.dtype == torch.float32 and records.dim() == 4):
+        raise ValueError("records must be a contiguous fp32 CUDA tensor [n_parts, B * H, n_text, d + 2]")
+    if not (out.is_cuda and out.is_contiguous() and out.dtype == torch.bfloat16 and out.dim() == 4):
+        raise ValueError("out must be a contiguous bf16 CUDA tensor [B, H, N, d]")
+    B, H, N, d = out.shape
+    if records.shape[1:] != (B * H, n_text, d + 2):
+        raise ValueError("records do not match out")
+    _check(load().clear_text_merge(records.data_ptr(), records.shape[0], B, H, n_text, d, mode, out.data_ptr(), N,
+                                   _stream_ptr(stream)), "clear_text_merge")
+    return out
 
 
 def clear_cache_clear() -> None:

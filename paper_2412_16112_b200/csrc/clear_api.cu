@@ -448,7 +448,59 @@ int clear_plan_mask_table(const clear_plan_t *plan, const uint32_t **words, int3
 int clear_attn_fwd_planned(const clear_plan_t *plan, const void *q, const void *k, const void *v, void *out,
                            float scale, void *stream)
 {
+    if (plan && plan->shape.part == CLEAR_PART_BAND_TEXT) return CLEAR_ERR_PLAN_MISMATCH;  // clear_attn_text_partial
     return forward(plan, q, k, v, out, scale, stream);
+}
+
+int clear_band_geometry(int grid_h, float radius, int mask_kind, int n_bands, int band, int32_t *y0, int32_t *y1,
+                        int32_t *halo_lo, int32_t *halo_hi)
+{
+    if (grid_h <= 0 || n_bands <= 0 || n_bands > grid_h || band < 0 || band >= n_bands) return CLEAR_ERR_INVALID_ARG;
+    if (!(radius > 0.f) || !std::isfinite(radius)) return CLEAR_ERR_INVALID_ARG;
+    if (mask_kind != CLEAR_MASK_DISC && mask_kind != CLEAR_MASK_SQUARE) return CLEAR_ERR_INVALID_ARG;
+    const int base = grid_h / n_bands, extra = grid_h % n_bands;
+    const int a = band * base + std::min(band, extra), b = a + base + (band < extra ? 1 : 0);
+    const int64_t reach = window_reach(radius, mask_kind);
+    if (y0) *y0 = a;
+    if (y1) *y1 = b;
+    if (halo_lo) *halo_lo = (int32_t)std::min<int64_t>(reach, a);
+    if (halo_hi) *halo_hi = (int32_t)std::min<int64_t>(reach, grid_h - b);
+    return CLEAR_OK;
+}
+
+int clear_plan_create_band(clear_plan_t **plan, int B, int H, int local_rows, int grid_w, int n_text, int head_dim,
+                           float radius, int mask_kind, int part, int q_row_begin, int q_row_end, int text_keys,
+                           int host_only)
+{
+    if (part != CLEAR_PART_BAND_IMAGE && part != CLEAR_PART_BAND_TEXT) return CLEAR_ERR_INVALID_ARG;
+    Shape s{B, H, local_rows, grid_w, n_text, head_dim, radius, CLEAR_BF16, CLEAR_KERNEL_TCGEN05_WS};
+    s.mask_kind = mask_kind;
+    s.part = part;
+    s.q_row_begin = q_row_begin;
+    s.q_row_end = q_row_end;
+    s.text_keys = text_keys != 0;
+    return create_plan(plan, s, host_only != 0);
+}
+
+int clear_attn_text_partial(const clear_plan_t *plan, const void *q, const void *k, const void *v, float *records,
+                            float scale, void *stream)
+{
+    if (!plan) return CLEAR_ERR_INVALID_ARG;
+    if (plan->shape.part != CLEAR_PART_BAND_TEXT) return CLEAR_ERR_PLAN_MISMATCH;
+    return forward(plan, q, k, v, records, scale, stream);
+}
+
+int clear_text_merge(const float *records, int n_parts, int B, int H, int n_text, int head_dim, int mode, void *out,
+                     long long out_tokens, void *stream)
+{
+    if (!records || !out || n_parts <= 0 || B <= 0 || H <= 0 || n_text <= 0 || out_tokens < n_text)
+        return CLEAR_ERR_INVALID_ARG;
+    if (mode != CLEAR_TEXT_MERGE_EXACT && mode != CLEAR_TEXT_MERGE_AVERAGE) return CLEAR_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return CLEAR_ERR_UNSUPPORTED;
+    if ((int64_t)B * H > 65535) return CLEAR_ERR_UNSUPPORTED;
+    if ((((uintptr_t)records) & 3u) || (((uintptr_t)out) & 15u)) return CLEAR_ERR_MISALIGNED;
+    return launch_text_merge(records, n_parts, B * H, n_text, head_dim, mode, out, out_tokens,
+                             static_cast<cudaStream_t>(stream));
 }
 
 int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_host, const void *v_host,
@@ -456,7 +508,7 @@ int clear_attn_fwd_host(clear_plan_t *plan, const void *q_host, const void *k_ho
 {
     if (!plan || !q_host || !k_host || !v_host || !out_host) return CLEAR_ERR_INVALID_ARG;
     if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
-    if (plan->host_only) return CLEAR_ERR_PLAN_MISMATCH;
+    if (plan->host_only || plan->shape.part != CLEAR_PART_ALL) return CLEAR_ERR_PLAN_MISMATCH;
     int dev = -1;
     CLEAR_CUDA_TRY(cudaGetDevice(&dev));
     if (dev != plan->device) return CLEAR_ERR_PLAN_MISMATCH;

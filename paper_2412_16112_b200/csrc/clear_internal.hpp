@@ -100,6 +100,11 @@ int launch_ws(const clear_plan &p, const void *q, const void *k, const void *v, 
 // fp32 backward pass on the CUDA cores (dk and dv are zeroed on the stream first).
 int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq,
                    void *dk, void *dv, float scale, cudaStream_t stream);
+// Row-band form: one (O, m, l) record per text row from a band-text plan's partial results, and the merge of the
+// records of all bands into bf16 text rows.
+int launch_text_export(const clear_plan &p, void *records, cudaStream_t stream);
+int launch_text_merge(const float *records, int n_parts, int n_bh, int n_text, int head_dim, int mode, void *out,
+                      long long out_tokens, cudaStream_t stream);
 // Q/K preparation (RMS normalisation, rotary embedding, factor on Q): one elementwise pass, no plan.
 int launch_qk_prep(const void *q_in, const void *k_in, void *q_out, void *k_out, const float *gain_q, const float *gain_k,
                    int n_bh, int grid_h, int grid_w, int n_text, int head_dim, int dtype, const int axes_dim[3],

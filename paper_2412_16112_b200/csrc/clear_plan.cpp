@@ -20,6 +20,14 @@ static int64_t isqrt64(int64_t v)
     return r;
 }
 
+int64_t window_reach(float radius, int mask_kind)
+{
+    const double r = (double)radius;
+    if (!(r < 1048576.0)) return 1048576;
+    if (mask_kind == CLEAR_MASK_SQUARE) return (int64_t)std::ceil(r) - 1;
+    return isqrt64((int64_t)std::ceil(r * r) - 1);
+}
+
 int validate_shape(const Shape &s)
 {
     if (s.B <= 0 || s.H <= 0 || s.grid_h <= 0 || s.grid_w <= 0 || s.n_text < 0 || s.head_dim <= 0)
@@ -28,6 +36,14 @@ int validate_shape(const Shape &s)
     if (s.dtype != CLEAR_BF16 && s.dtype != CLEAR_F32) return CLEAR_ERR_INVALID_ARG;
     if (s.kernel < CLEAR_KERNEL_AUTO || s.kernel > CLEAR_KERNEL_TCGEN05_WS) return CLEAR_ERR_INVALID_ARG;
     if (s.mask_kind != CLEAR_MASK_DISC && s.mask_kind != CLEAR_MASK_SQUARE) return CLEAR_ERR_INVALID_ARG;
+    if (s.part != CLEAR_PART_ALL) {
+        if (s.part != CLEAR_PART_BAND_IMAGE && s.part != CLEAR_PART_BAND_TEXT) return CLEAR_ERR_INVALID_ARG;
+        if (s.q_row_begin < 0 || s.q_row_end <= s.q_row_begin || s.q_row_end > s.grid_h) return CLEAR_ERR_INVALID_ARG;
+        if (s.part == CLEAR_PART_BAND_TEXT && s.n_text <= 0) return CLEAR_ERR_INVALID_ARG;
+        // band parts exist for the warp-specialised tensor-core kernel only
+        if (s.kernel != CLEAR_KERNEL_AUTO && s.kernel != CLEAR_KERNEL_TCGEN05_WS) return CLEAR_ERR_UNSUPPORTED;
+        if (s.dtype != CLEAR_BF16 || (s.head_dim != 64 && s.head_dim != 128)) return CLEAR_ERR_UNSUPPORTED;
+    }
     const int64_t n = (int64_t)s.grid_h * s.grid_w;
     const int64_t N = n + s.n_text;
     if (N > (int64_t)1 << 30) return CLEAR_ERR_UNSUPPORTED;  // token indices stay in int32
@@ -226,6 +242,22 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
     const int gh = s.grid_h, gw = s.grid_w, T = s.n_text;
     const int64_t N = (int64_t)gh * gw + T;
     const int R = (int)sch.half_width.size() - 1;  // rows a window reaches up and down
+    if (s.part == CLEAR_PART_BAND_IMAGE) {
+        // allowed pairs of the band's image queries: the text keys, and per row offset the closed form
+        // sum_x (min(x+m, gw-1) - max(x-m, 0) + 1) for the rows that are on this grid
+        int64_t pairs = 0;
+        for (int64_t y = s.q_row_begin; y < s.q_row_end; ++y) {
+            pairs += (int64_t)gw * T;
+            for (int64_t dy = -R; dy <= R; ++dy) {
+                if (y + dy < 0 || y + dy >= gh) continue;
+                const int64_t m = sch.half_width[(size_t)(dy < 0 ? -dy : dy)];
+                pairs += (int64_t)gw * (2 * m + 1) - m * (m + 1);
+            }
+        }
+        sch.sum_mask = pairs;
+    } else if (s.part == CLEAR_PART_BAND_TEXT) {
+        sch.sum_mask = (int64_t)T * ((s.text_keys ? T : 0) + (int64_t)(s.q_row_end - s.q_row_begin) * gw);
+    }
 
     sch.pair_items.clear();
     sch.pair_steps.clear();
@@ -290,17 +322,32 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
         sch.pair_steps.push_back(st);
     };
 
-    // ---- text-query tiles, two per item, dense over all N keys, split over key ranges ----------
-    const int n_lin = (int)((N + kTileTokens - 1) / kTileTokens);
-    sch.n_text_tiles = (T + kTileTokens - 1) / kTileTokens;
+    // ---- text-query tiles, two per item, dense over their keys, split over key ranges ----------
+    // The keys of a text query as runs of tokens: all N of them; for the text part of a band, the text tokens
+    // (if this band counts them) and the image tokens of the band's own rows.
+    std::vector<std::pair<int64_t, int64_t>> key_runs;
+    if (s.part == CLEAR_PART_ALL) {
+        key_runs.push_back({0, N});
+    } else if (s.part == CLEAR_PART_BAND_TEXT) {
+        if (s.text_keys) key_runs.push_back({0, T});
+        key_runs.push_back({T + (int64_t)s.q_row_begin * gw, T + (int64_t)s.q_row_end * gw});
+    }
+    std::vector<std::pair<int, int>> lin_tiles;  // first token, tokens that count
+    for (const auto &run : key_runs)
+        for (int64_t t0 = run.first; t0 < run.second; t0 += kTileTokens)
+            lin_tiles.push_back({(int)t0, (int)std::min<int64_t>(kTileTokens, run.second - t0)});
+    const int n_lin = (int)lin_tiles.size();
+    sch.n_text_tiles = n_lin > 0 ? (T + kTileTokens - 1) / kTileTokens : 0;
     int chunk = n_lin, n_splits = 1;
     if (sch.n_text_tiles > 0) {
         n_splits = (n_lin + kSplitTargetTiles - 1) / kSplitTargetTiles;
         chunk = (n_lin + n_splits - 1) / n_splits;
         n_splits = (n_lin + chunk - 1) / chunk;
     }
+    // the text part of a band always leaves partial results (they are merged with the other bands')
+    const bool partials = n_splits > 1 || s.part == CLEAR_PART_BAND_TEXT;
     sch.n_text_splits = sch.n_text_tiles > 0 ? n_splits : 0;
-    sch.n_partial_slots = (sch.n_text_tiles > 0 && n_splits > 1) ? sch.n_text_tiles * n_splits : 0;
+    sch.n_partial_slots = (sch.n_text_tiles > 0 && partials) ? sch.n_text_tiles * n_splits : 0;
     // key range outermost: the items that stream one key range sit next to each other in the queue
     for (int sp = 0; sp < n_splits && sch.n_text_tiles > 0; ++sp) {
         for (int tq = 0; tq < sch.n_text_tiles; tq += 2) {
@@ -312,19 +359,26 @@ void build_pair_schedule(const Shape &s, Schedule &sch)
             it.n_rows1 = it.n_sides == 2 ? std::min(kTileTokens, T - it.qx - kTileTokens) : 0;
             it.step_begin = (int32_t)sch.pair_steps.size();
             const int t0 = sp * chunk, t1 = std::min(n_lin, t0 + chunk);
-            for (int t = t0; t < t1; ++t)
-                linear_step(t * kTileTokens, (int)std::min<int64_t>(kTileTokens, N - (int64_t)t * kTileTokens),
-                            it.n_sides);
-            it.partial_slot0 = n_splits > 1 ? tq * n_splits + sp : -1;
-            it.partial_slot1 = (n_splits > 1 && it.n_sides == 2) ? (tq + 1) * n_splits + sp : -1;
+            for (int t = t0; t < t1; ++t) linear_step(lin_tiles[(size_t)t].first, lin_tiles[(size_t)t].second, it.n_sides);
+            it.partial_slot0 = partials ? tq * n_splits + sp : -1;
+            it.partial_slot1 = (partials && it.n_sides == 2) ? (tq + 1) * n_splits + sp : -1;
             finish_item(it);
         }
     }
     sch.n_text_pair_items = (int)sch.pair_items.size();
 
     // ---- image-query patches, two vertically adjacent ones per item ----------------------------
-    const int ntx = (gw + kTileW - 1) / kTileW, nty = (gh + kTileH - 1) / kTileH;
-    for (int ty = 0; ty < nty; ty += 2) {
+    // (of a band: the patches that hold rows of the band; rows of those patches outside the band are computed
+    // and written too, which the caller of a band part is told)
+    const int ntx = (gw + kTileW - 1) / kTileW;
+    int ty_begin = 0, nty = (gh + kTileH - 1) / kTileH;
+    if (s.part == CLEAR_PART_BAND_IMAGE) {
+        ty_begin = s.q_row_begin / kTileH;
+        nty = (s.q_row_end + kTileH - 1) / kTileH;
+    } else if (s.part == CLEAR_PART_BAND_TEXT) {
+        nty = 0;
+    }
+    for (int ty = ty_begin; ty < nty; ty += 2) {
         for (int tx = 0; tx < ntx; ++tx) {
             clear_pair_item_t it{};
             it.kind = 0;

@@ -20,11 +20,17 @@ struct Shape {
     int dtype = 0;
     int kernel = 0;
     int mask_kind = 0;  // CLEAR_MASK_DISC (Eq. 3) or CLEAR_MASK_SQUARE
+    // Row-band parallel form (Sec. 3.4): the grid of this shape is a band of image rows with the halo rows around
+    // it; `part` selects what the plan computes of it (CLEAR_PART_*).
+    int part = 0;
+    int q_row_begin = 0, q_row_end = 0;  // rows of the band inside the grid (band parts only)
+    int text_keys = 1;                   // CLEAR_PART_BAND_TEXT: are the text tokens among the keys
     bool operator==(const Shape &o) const
     {
         return B == o.B && H == o.H && grid_h == o.grid_h && grid_w == o.grid_w && n_text == o.n_text &&
                head_dim == o.head_dim && radius == o.radius && dtype == o.dtype && kernel == o.kernel &&
-               mask_kind == o.mask_kind;
+               mask_kind == o.mask_kind && part == o.part && q_row_begin == o.q_row_begin &&
+               q_row_end == o.q_row_end && text_keys == o.text_keys;
     }
 };
 
@@ -45,6 +51,9 @@ struct Schedule {
     int64_t sum_mask = 0;
     int64_t executed_pairs = 0;
 };
+
+// Largest row offset |dy| at which the window lets an image query see a key on an unbounded grid (capped at 2^20).
+int64_t window_reach(float radius, int mask_kind);
 
 // Validate the arguments every entry point shares.  Returns a clear_status.
 int validate_shape(const Shape &s);

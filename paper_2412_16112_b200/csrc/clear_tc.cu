@@ -478,6 +478,8 @@ int launch_variant(const clear_plan &p, const CUtensorMap *tm, const TcParams &p
 int launch_text_combine(const clear_plan &p, void *out, cudaStream_t stream)
 {
     const Shape &s = p.shape;
+    // the text part of a band leaves records for the merge over all bands instead of finished rows
+    if (s.part == CLEAR_PART_BAND_TEXT) return launch_text_export(p, out, stream);
     if (p.sch.n_partial_slots <= 0) return CLEAR_OK;
     const int64_t N = (int64_t)s.n_text + (int64_t)s.grid_h * s.grid_w;
     dim3 cgrid((unsigned)s.n_text, (unsigned)(s.B * s.H));
