@@ -417,6 +417,92 @@ def run_ours(args, w):
     return 0
 
 
+def run_bands(args, w):
+    """`--parallelism bands`: ONE workload cut into row bands over the ranks (Sec. 3.4): halo exchange, the band's
+    image queries, the text queries' records, all-gather and merge, all inside the timed region.  Strong scaling;
+    `value` = the whole workload's flops over the slowest rank's time.  Local inputs are drawn on the device."""
+    from paper_2412_16112_b200 import band_parallel as bp
+    from paper_2412_16112_b200 import binding as clear
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    if w.dtype != "bf16":
+        raise RuntimeError("row bands exist for the bf16 workloads")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    peaks, peaks_kind = load_peaks()
+    att = bp.BandAttention(w.B, w.H, w.grid_h, w.grid_w, w.n_text, w.head_dim, w.radius, rank, world,
+                           text_mode="average" if args.text_mode == "average" else "exact")
+    lay = att.lay
+    gen = torch.Generator(device=dev).manual_seed(w.seed + 100 * rank)
+    shape = (w.B, w.H, lay.n_local_tokens, w.head_dim)
+
+    def draw(norm):
+        x = torch.randn(shape, generator=gen, device=dev, dtype=torch.float32)
+        if norm:
+            x = x / torch.sqrt(x.pow(2).mean(dim=-1, keepdim=True) + 1e-6)
+        return x.to(torch.bfloat16)
+    qd, kd, vd = draw(True), draw(True), draw(False)
+    out = torch.empty_like(qd)
+    stream = torch.cuda.current_stream()
+    whole = clear.Plan(w.B, w.H, w.grid_h, w.grid_w, w.n_text, w.head_dim, w.radius, host_only=True).info()
+    flops = whole.flops
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    att.forward(qd, kd, vd, out, w.scale)
+    w0.record(stream)
+    for _ in range(args.warmup):
+        att.forward(qd, kd, vd, out, w.scale)
+    w1.record(stream)
+    att.check()
+    if args.steps is None:
+        warm_ms = max_over_ranks(w0.elapsed_time(w1) / args.warmup, dist, dev)
+        args.steps = int(min(2000, max(20, math.ceil(600.0 / max(warm_ms, 1e-3)))))
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        for s in range(args.steps):
+            ev[s][0].record(stream)
+            att.forward(qd, kd, vd, out, w.scale)
+            ev[s][1].record(stream)
+        barrier()
+    att.check()
+    ms = [a.elapsed_time(b) for a, b in ev]
+    ms_per_step = max_over_ranks(float(sum(ms)), dist, dev) / args.steps
+    if rank == 0:
+        value = flops / (ms_per_step * 1e-3) / 1e12
+        peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+        halo_bytes = 2 * (lay.halo_lo + lay.halo_hi) * w.grid_w * w.head_dim * 2 * w.B * w.H
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic (drawn on the device, per rank)",
+                "config": dict(workload_config(w), parallelism=f"row bands x{world}", text_rows=args.text_mode,
+                               l2="local tensors larger than L2" if 4 * qd.numel() * 2 > 2 * 126e6 else "local tensors fit in L2"),
+                "clocks": clocks.summary(), "e2e": None, "gpu_launches": 4 * args.steps,
+                "roofline": {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s",
+                             "frac": value / world / peak, "traffic": None, "peak_kind": f"{peaks_kind} bf16 burst",
+                             "kernel": "clear_ws_kernel (band image plan + band text plan) + export and merge kernels"},
+                "cpu_baseline": None, "flops_per_call": flops, "parallelism": "row bands",
+                "halo_bytes_received_rank0": halo_bytes,
+                "record_bytes_gathered": world * w.B * w.H * w.n_text * (w.head_dim + 2) * 4}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -428,11 +514,18 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-prep", action="store_true", help="skip the timing of the Q/K preparation kernel")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--parallelism", default="replicas", choices=["replicas", "bands"],
+                    help="replicas (default): every rank runs the whole workload; bands: one workload cut into row "
+                         "bands over the ranks (Sec. 3.4), strong scaling")
+    ap.add_argument("--text-mode", default="exact", choices=["exact", "average"],
+                    help="bands: exact merge of the text rows, or the patch-wise average of Eq. 7")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = workloads.WORKLOADS[args.workload]
     if args.impl == "reference":
         return run_reference(args, w)
+    if args.parallelism == "bands":
+        return run_bands(args, w)
     return run_ours(args, w)
 
 
