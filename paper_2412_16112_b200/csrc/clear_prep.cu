@@ -3,7 +3,7 @@
 // constant factor folded into Q (the log-scale attention factor of Sec. 4.3's high-resolution recipe).
 //
 // The work is elementwise with one reduction per row of d channels, so HBM bounds it: every element of Q and
-// K is read once and written once (4 * B * H * N * d * sizeof(element) bytes per call).  One warp owns one
+// K is read once and written once (4 * B * H * N * d * sizeof(element) bytes per call).  One warp owns a
 // few token positions (32 / (d / 8) of them) and walks over all (batch, head) rows of those tokens: the angles
 // depend on the position only, so their sines and cosines are computed once per token and reused for
 // 2 * B * H rows; a lane holds 8 consecutive channels of a row (whole rotary pairs), so a row is one
