@@ -211,8 +211,13 @@ float clear_log_scale_factor(long long n_tokens, long long n_train_tokens);
 /* Window of an image query (text tokens are always allowed, as in Eq. 3). */
 enum {
     CLEAR_MASK_DISC = 0,   /* Eq. 3: dx^2 + dy^2 < r^2, the paper's circular window                              */
-    CLEAR_MASK_SQUARE = 1  /* max(|dx|, |dy|) < r: the square sliding window of Neighborhood Attention, which
+    CLEAR_MASK_SQUARE = 1, /* max(|dx|, |dy|) < r: the square sliding window of Neighborhood Attention, which
                               Sec. 3.2 sets the circular one against (the circle costs about pi / 4 of it)      */
+    CLEAR_MASK_WINDOWS = 2, /* both tokens in the same w x w window of the grid, the window grid shifted by s
+                               (floor((x + s) / w) and floor((y + s) / w) agree; no wrap-around): the Swin baseline
+                               of the appendix (w = 16, s = 8 in every other layer)                              */
+    CLEAR_MASK_STRIDED = 3  /* (xj - xi) mod r == l mod r and (yj - yi) mod r == (l div r) mod r, non-negative
+                               remainders: the strided baseline of the appendix at layer l                      */
 };
 
 /* Build the schedule for one shape on the current device (Eq. 3 turned into integer geometry):
@@ -294,6 +299,18 @@ int clear_attn_text_partial(const clear_plan_t *plan, const void *q, const void 
  * Errors: INVALID_ARG, UNSUPPORTED (head_dim other than 64 or 128, B * H > 65535), MISALIGNED, CUDA. */
 int clear_text_merge(const float *records, int n_parts, int B, int H, int n_text, int head_dim, int mode, void *out,
                      long long out_tokens, void *stream);
+
+/* Plan for any mask kind (bf16 or fp32).  mask_size: r of CLEAR_MASK_DISC / CLEAR_MASK_SQUARE, the window size w
+ * of CLEAR_MASK_WINDOWS, the stride r of CLEAR_MASK_STRIDED (the last two whole numbers >= 1); mask_param: the shift
+ * s of the window grid, the layer index l of the strided mask, 0 for the other kinds.  The windows and the strided
+ * mask are no windows around the query (membership depends on absolute position, or on a residue class), so the
+ * tensor-core kernels' tables do not carry them: these two kinds run on the fp32-accumulating CUDA-core kernel,
+ * which walks the allowed keys of each query row by row (the kernel is chosen by the library).  They serve to
+ * reproduce the appendix's comparison masks; clear_plan_info reports their sum(M) and flops.
+ * Run the plan with clear_attn_fwd_planned.  Errors as clear_plan_create_ex; INVALID_ARG for a fractional window
+ * size or stride, a negative shift or layer, a non-zero mask_param with the disc or the square. */
+int clear_plan_create_mask(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, int dtype,
+                           int mask_kind, float mask_size, int mask_param, int host_only);
 
 /* The same schedule built on the host only: no CUDA call is made and no device is needed.  The
  * plan can be inspected (clear_plan_info, clear_plan_tables) and destroyed, not executed

@@ -18,7 +18,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_PLAN_MISMATCH = -1, -2, -3
 ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_NO_MEMORY, ERR_TOO_LARGE = -5, -6, -7, -8
 BF16, F32 = 0, 1
 KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_TCGEN05_WS = 0, 1, 2, 3
-MASK_DISC, MASK_SQUARE = 0, 1
+MASK_DISC, MASK_SQUARE, MASK_WINDOWS, MASK_STRIDED = 0, 1, 2, 3
 PART_ALL, PART_BAND_IMAGE, PART_BAND_TEXT = 0, 1, 2
 TEXT_MERGE_EXACT, TEXT_MERGE_AVERAGE = 0, 1
 TILE_LINEAR, TILE_MASKED = 1, 2
@@ -33,6 +33,7 @@ EXPORTS = [
     "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim", "clear_attn_bwd_f32", "clear_plan_create_ex",
     "clear_qk_norm_rope", "clear_log_scale_factor",
     "clear_band_geometry", "clear_plan_create_band", "clear_attn_text_partial", "clear_text_merge",
+    "clear_plan_create_mask",
 ]
 
 
@@ -103,6 +104,7 @@ def load() -> ctypes.CDLL:
         lib.clear_plan_create_band.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, f32, i32, i32, i32, i32,
                                                i32, i32]
         lib.clear_attn_text_partial.argtypes = [vp, vp, vp, vp, vp, f32, vp]
+        lib.clear_plan_create_mask.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, i32, i32, f32, i32, i32]
         lib.clear_text_merge.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, ctypes.c_longlong, vp]
         lib.clear_log_scale_factor.argtypes = [ctypes.c_longlong, ctypes.c_longlong]
         lib.clear_log_scale_factor.restype = f32
@@ -255,9 +257,17 @@ class Plan:
     """Owner of a ``clear_plan_t``."""
 
     def __init__(self, B, H, grid_h, grid_w, n_text, head_dim, radius, dtype=BF16, kernel=KERNEL_AUTO,
-                 host_only=False, mask_kind=MASK_DISC):
+                 host_only=False, mask_kind=MASK_DISC, mask_param=0):
+        """``radius``: r of the disc / square window, the window size of ``MASK_WINDOWS``, the stride of
+        ``MASK_STRIDED``; ``mask_param``: the shift of the window grid / the layer index of the strided mask."""
         self._h = ctypes.c_void_p()
-        if mask_kind != MASK_DISC:
+        if mask_kind in (MASK_WINDOWS, MASK_STRIDED) or mask_param != 0:
+            if kernel not in (KERNEL_AUTO, KERNEL_SIMT):
+                raise ClearError(ERR_UNSUPPORTED, "clear_plan_create_mask")
+            _check(load().clear_plan_create_mask(ctypes.byref(self._h), B, H, grid_h, grid_w, n_text, head_dim, dtype,
+                                                 mask_kind, float(radius), mask_param, 1 if host_only else 0),
+                   "clear_plan_create_mask")
+        elif mask_kind != MASK_DISC:
             _check(load().clear_plan_create_ex(ctypes.byref(self._h), B, H, grid_h, grid_w, n_text, head_dim,
                                                float(radius), dtype, kernel, mask_kind, 1 if host_only else 0),
                    "clear_plan_create_ex")

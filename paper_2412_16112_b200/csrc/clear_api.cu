@@ -19,6 +19,7 @@ namespace {
 int select_kernel(const Shape &s)
 {
     if (s.kernel != CLEAR_KERNEL_AUTO) return s.kernel;
+    if (s.mask_kind == CLEAR_MASK_WINDOWS || s.mask_kind == CLEAR_MASK_STRIDED) return CLEAR_KERNEL_SIMT;
     if (s.dtype == CLEAR_BF16 && (s.head_dim == 64 || s.head_dim == 128)) return CLEAR_KERNEL_TCGEN05_WS;
     return CLEAR_KERNEL_SIMT;
 }
@@ -402,6 +403,15 @@ int clear_plan_create_ex(clear_plan_t **plan, int B, int H, int grid_h, int grid
 {
     Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, dtype, kernel};
     s.mask_kind = mask_kind;
+    return create_plan(plan, s, host_only != 0);
+}
+
+int clear_plan_create_mask(clear_plan_t **plan, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, int dtype,
+                           int mask_kind, float mask_size, int mask_param, int host_only)
+{
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, mask_size, dtype, CLEAR_KERNEL_AUTO};
+    s.mask_kind = mask_kind;
+    s.mask_param = mask_param;
     return create_plan(plan, s, host_only != 0);
 }
 

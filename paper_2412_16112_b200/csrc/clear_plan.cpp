@@ -35,7 +35,17 @@ int validate_shape(const Shape &s)
     if (!(s.radius > 0.f) || !std::isfinite(s.radius)) return CLEAR_ERR_INVALID_ARG;
     if (s.dtype != CLEAR_BF16 && s.dtype != CLEAR_F32) return CLEAR_ERR_INVALID_ARG;
     if (s.kernel < CLEAR_KERNEL_AUTO || s.kernel > CLEAR_KERNEL_TCGEN05_WS) return CLEAR_ERR_INVALID_ARG;
-    if (s.mask_kind != CLEAR_MASK_DISC && s.mask_kind != CLEAR_MASK_SQUARE) return CLEAR_ERR_INVALID_ARG;
+    if (s.mask_kind < CLEAR_MASK_DISC || s.mask_kind > CLEAR_MASK_STRIDED) return CLEAR_ERR_INVALID_ARG;
+    if (s.mask_kind == CLEAR_MASK_WINDOWS || s.mask_kind == CLEAR_MASK_STRIDED) {
+        // window size / stride: a whole number of grid cells; shift / layer index: not negative
+        if (s.radius < 1.f || s.radius != std::floor(s.radius) || s.radius > 1048576.f || s.mask_param < 0)
+            return CLEAR_ERR_INVALID_ARG;
+        // masks that are no window around the query run on the CUDA-core kernel only, and not as band parts
+        if (s.kernel != CLEAR_KERNEL_AUTO && s.kernel != CLEAR_KERNEL_SIMT) return CLEAR_ERR_UNSUPPORTED;
+        if (s.part != CLEAR_PART_ALL) return CLEAR_ERR_UNSUPPORTED;
+    } else if (s.mask_param != 0) {
+        return CLEAR_ERR_INVALID_ARG;
+    }
     if (s.part != CLEAR_PART_ALL) {
         if (s.part != CLEAR_PART_BAND_IMAGE && s.part != CLEAR_PART_BAND_TEXT) return CLEAR_ERR_INVALID_ARG;
         if (s.q_row_begin < 0 || s.q_row_end <= s.q_row_begin || s.q_row_end > s.grid_h) return CLEAR_ERR_INVALID_ARG;
@@ -59,10 +69,42 @@ int validate_shape(const Shape &s)
     return CLEAR_OK;
 }
 
+// Allowed (query, key) pairs along one axis of `len` cells for the two masks that factor over the axes.
+static int64_t axis_pairs(const Shape &s, int64_t len, bool y_axis)
+{
+    const int64_t a = (int64_t)s.radius;
+    int64_t pairs = 0;
+    if (s.mask_kind == CLEAR_MASK_WINDOWS) {
+        // cells c with the same floor((c + shift) / w) share a window: segments of the axis, squared
+        const int64_t shift = s.mask_param;
+        int64_t c = 0;
+        while (c < len) {
+            const int64_t end = std::min(len, ((c + shift) / a + 1) * a - shift);
+            pairs += (end - c) * (end - c);
+            c = end;
+        }
+    } else {
+        // strided: key = query + offset (mod stride), offset = layer % stride (x) or (layer / stride) % stride (y)
+        const int64_t off = y_axis ? (s.mask_param / a) % a : s.mask_param % a;
+        for (int64_t c = 0; c < len; ++c) {
+            const int64_t first = (c + off) % a;  // smallest cell congruent to c + off
+            if (first < len) pairs += (len - 1 - first) / a + 1;
+        }
+    }
+    return pairs;
+}
+
 void build_geometry(const Shape &s, Schedule &sch)
 {
     const int64_t gh = s.grid_h, gw = s.grid_w, T = s.n_text;
     const int64_t n = gh * gw, N = n + T;
+    if (s.mask_kind == CLEAR_MASK_WINDOWS || s.mask_kind == CLEAR_MASK_STRIDED) {
+        // no window around the query: no half widths; the mask factors into a row rule and a column rule
+        sch.thr = 0;
+        sch.half_width.clear();
+        sch.sum_mask = T * N + n * T + axis_pairs(s, gh, true) * axis_pairs(s, gw, false);
+        return;
+    }
     // Eq. 3 with integer squared distances: d2 < r^2  <=>  d2 < ceil(r^2).  No pair on the grid
     // is farther apart than its diagonal, so the threshold is capped just above it.
     const double r = (double)s.radius;

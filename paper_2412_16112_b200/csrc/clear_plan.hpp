@@ -19,7 +19,8 @@ struct Shape {
     float radius = 0.f;
     int dtype = 0;
     int kernel = 0;
-    int mask_kind = 0;  // CLEAR_MASK_DISC (Eq. 3) or CLEAR_MASK_SQUARE
+    int mask_kind = 0;  // CLEAR_MASK_*: `radius` is r of the disc / square, the window size, or the stride
+    int mask_param = 0; // CLEAR_MASK_WINDOWS: shift of the window grid; CLEAR_MASK_STRIDED: layer index
     // Row-band parallel form (Sec. 3.4): the grid of this shape is a band of image rows with the halo rows around
     // it; `part` selects what the plan computes of it (CLEAR_PART_*).
     int part = 0;
@@ -29,7 +30,7 @@ struct Shape {
     {
         return B == o.B && H == o.H && grid_h == o.grid_h && grid_w == o.grid_w && n_text == o.n_text &&
                head_dim == o.head_dim && radius == o.radius && dtype == o.dtype && kernel == o.kernel &&
-               mask_kind == o.mask_kind && part == o.part && q_row_begin == o.q_row_begin &&
+               mask_kind == o.mask_kind && mask_param == o.mask_param && part == o.part && q_row_begin == o.q_row_begin &&
                q_row_end == o.q_row_end && text_keys == o.text_keys;
     }
 };

@@ -5,6 +5,8 @@
 // scales.  Each warp walks the keys its query may see under Eq. 3 -- the text tokens, then for
 // every grid row within reach the run of columns [x - m(dy), x + m(dy)] clipped to the grid --
 // and keeps an online softmax (Eq. 1) over blocks of 8 keys.  Lanes split the head dimension.
+// The two comparison masks of the appendix that are no window around the query run here too: the
+// shifted window grid (a rectangle of keys per query) and the strided mask (every r-th row and column).
 #include <cuda_bf16.h>
 
 #include "clear_internal.hpp"
@@ -24,7 +26,7 @@ template <typename T, int EPL>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 clear_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v, T *__restrict__ out,
                   int grid_h, int grid_w, int n_text, int d, const int32_t *__restrict__ half_width, int n_half_width,
-                  float scale)
+                  int mask_kind, int mask_size, int mask_param, float scale)
 {
     const int lane = threadIdx.x & 31;
     const int64_t N = (int64_t)n_text + (int64_t)grid_h * grid_w;
@@ -41,13 +43,13 @@ clear_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__r
     }
     float m = -INFINITY, l = 0.f;
 
-    // online softmax over the tokens [j0, j1)
-    auto run = [&](int64_t j0, int64_t j1) {
-        for (int64_t j = j0; j < j1; j += kKeyBlock) {
+    // online softmax over the tokens j0, j0 + step, ... below j1
+    auto run = [&](int64_t j0, int64_t j1, int64_t step) {
+        for (int64_t j = j0; j < j1; j += kKeyBlock * step) {
             float s[kKeyBlock];
 #pragma unroll
             for (int u = 0; u < kKeyBlock; ++u) {
-                const int64_t jj = j + u;
+                const int64_t jj = j + u * step;
                 float part = 0.f;
                 if (jj < j1) {
 #pragma unroll
@@ -62,7 +64,7 @@ clear_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__r
             for (int u = 0; u < kKeyBlock; ++u) {
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
-                if (j + u >= j1) s[u] = -INFINITY;
+                if (j + u * step >= j1) s[u] = -INFINITY;
             }
             float m_new = m;
 #pragma unroll
@@ -73,7 +75,7 @@ clear_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__r
             for (int t = 0; t < EPL; ++t) acc[t] *= alpha;
 #pragma unroll
             for (int u = 0; u < kKeyBlock; ++u) {
-                const int64_t jj = j + u;
+                const int64_t jj = j + u * step;
                 if (jj < j1) {
                     const float p = expf(s[u] - m_new);
                     l += p;
@@ -89,23 +91,44 @@ clear_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__r
     };
 
     if (i < n_text) {
-        run(0, N);  // a text query sees every token
+        run(0, N, 1);  // a text query sees every token
     } else {
-        run(0, n_text);  // every image query sees all text keys
+        run(0, n_text, 1);  // every image query sees all text keys
         const int64_t pix = i - n_text;
         const int y = (int)(pix / grid_w), x = (int)(pix % grid_w);
-        const int R = n_half_width - 1;
-        for (int dy = -R; dy <= R; ++dy) {
-            const int yy = y + dy;
-            if (yy < 0 || yy >= grid_h) continue;
-            const int hw = half_width[dy < 0 ? -dy : dy];
-            const int lo = max(x - hw, 0), hi = min(x + hw, grid_w - 1);
-            const int64_t row0 = (int64_t)n_text + (int64_t)yy * grid_w;
-            run(row0 + lo, row0 + hi + 1);
+        if (mask_kind == CLEAR_MASK_WINDOWS) {
+            // the w x w window of the shifted window grid that holds (y, x), clipped to the grid
+            const int w = mask_size, sh = mask_param;
+            const int y_lo = max(((y + sh) / w) * w - sh, 0), y_hi = min(((y + sh) / w + 1) * w - sh, grid_h);
+            const int x_lo = max(((x + sh) / w) * w - sh, 0), x_hi = min(((x + sh) / w + 1) * w - sh, grid_w);
+            for (int yy = y_lo; yy < y_hi; ++yy) {
+                const int64_t row0 = (int64_t)n_text + (int64_t)yy * grid_w;
+                run(row0 + x_lo, row0 + x_hi, 1);
+            }
+        } else if (mask_kind == CLEAR_MASK_STRIDED) {
+            // rows congruent to y + (l div r), columns congruent to x + (l mod r), modulo the stride r
+            const int r = mask_size;
+            const int y0 = (y + (mask_param / r) % r) % r, x0 = (x + mask_param % r) % r;
+            for (int yy = y0; yy < grid_h; yy += r) {
+                const int64_t row0 = (int64_t)n_text + (int64_t)yy * grid_w;
+                run(row0 + x0, row0 + grid_w, r);
+            }
+        } else {
+            const int R = n_half_width - 1;
+            for (int dy = -R; dy <= R; ++dy) {
+                const int yy = y + dy;
+                if (yy < 0 || yy >= grid_h) continue;
+                const int hw = half_width[dy < 0 ? -dy : dy];
+                const int lo = max(x - hw, 0), hi = min(x + hw, grid_w - 1);
+                const int64_t row0 = (int64_t)n_text + (int64_t)yy * grid_w;
+                run(row0 + lo, row0 + hi + 1, 1);
+            }
         }
     }
 
-    const float inv = 1.f / l;  // l >= 1: the query itself (image) or any token (text) is always allowed
+    // l > 0: an image query sees itself under the disc, the square and the windows, and the text keys always;
+    // under the strided mask with no text a query may see nothing: its output is 0
+    const float inv = l > 0.f ? 1.f / l : 0.f;
 #pragma unroll
     for (int t = 0; t < EPL; ++t) {
         const int e = lane + 32 * t;
@@ -127,7 +150,8 @@ int launch_typed(const clear_plan &p, const void *q, const void *k, const void *
     case E:                                                                                                     \
         clear_simt_kernel<T, E><<<grid, block, 0, stream>>>((const T *)q, (const T *)k, (const T *)v, (T *)out, \
                                                             s.grid_h, s.grid_w, s.n_text, s.head_dim,           \
-                                                            p.d_half_width, n_hw, scale);                       \
+                                                            p.d_half_width, n_hw, s.mask_kind, (int)s.radius,   \
+                                                            s.mask_param, scale);                               \
         break;
     switch (epl) {
         CLEAR_SIMT_CASE(1)

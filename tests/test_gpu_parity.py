@@ -601,3 +601,40 @@ def test_square_window_matches_its_oracle(kernel, gh, gw, T, r):
     disc = oracle.attn(q, k, v, gh, gw, T, r, scale)
     assert np.abs(want - disc).max() > 1e-3
     plan.destroy()
+
+
+# ----------------------------------------------------------------------------------------------
+# the appendix's comparison masks that are no window around the query (CUDA-core kernel)
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("kind,a,b,gh,gw,T", [
+    ("windows", 16, 0, 40, 48, 130),    # the Swin baseline's window size, aligned grid of windows
+    ("windows", 16, 8, 40, 48, 130),    # shifted by half a window: cut windows at every border
+    ("windows", 5, 2, 13, 19, 7),       # sizes that divide nothing
+    ("windows", 4, 0, 9, 33, 0),        # no text
+    ("strided", 4, 0, 24, 40, 130),     # layer 0: every fourth row and column from the query's own
+    ("strided", 4, 6, 24, 40, 130),     # layer 6: offset (2, 1)
+    ("strided", 7, 30, 13, 19, 7),
+    ("strided", 3, 4, 10, 10, 0),       # no text: queries near the border still see a key of their class
+])
+def test_window_grid_and_strided_masks_match_their_oracle(dtype, kind, a, b, gh, gw, T):
+    from oracle import clear_oracle_windows as win
+    d = 64
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, dtype=dtype, qk_norm=dtype == "bf16", seed=gh * 5 + gw + b)
+    scale = 1 / math.sqrt(d)
+    okind = win.WINDOWS if kind == "windows" else win.STRIDED
+    ckind = clear.MASK_WINDOWS if kind == "windows" else clear.MASK_STRIDED
+    want = win.attn(q, k, v, gh, gw, T, okind, a, b, scale)
+    plan = clear.Plan(1, 2, gh, gw, T, d, a, dtype=clear.BF16 if dtype == "bf16" else clear.F32, mask_kind=ckind, mask_param=b)
+    info = plan.info()
+    assert info.kernel == clear.KERNEL_SIMT and info.sum_mask == win.mask_counts(okind, a, b, gh, gw, T)[0]
+    qd, kd, vd = (t.to(dev()) for t in (q, k, v))
+    out = torch.full_like(qd, float("nan"))
+    plan.forward(qd, kd, vd, out, scale)
+    plan.check()
+    if dtype == "bf16":
+        assert_close_bf16(out.cpu(), want, f"{kind} {a} {b}")
+    else:
+        err = np.abs(out.cpu().to(torch.float64).numpy() - want)
+        assert err.max() <= 1e-5, float(err.max())
+    plan.destroy()

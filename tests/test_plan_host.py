@@ -432,3 +432,48 @@ def test_square_window_geometry_and_schedules(gh, gw, T, r):
                 assert not (row & ~covered).any()
     with pytest.raises(clear.ClearError):
         clear.Plan(1, 1, gh, gw, T, 128, r, host_only=True, mask_kind=5)
+
+
+@pytest.mark.parametrize("kind,a,b,gh,gw,T", [
+    ("windows", 16, 0, 64, 64, 512), ("windows", 16, 8, 64, 64, 512), ("windows", 5, 2, 13, 19, 7),
+    ("windows", 100, 3, 9, 11, 0), ("strided", 4, 0, 64, 64, 512), ("strided", 4, 5, 20, 13, 3),
+    ("strided", 7, 30, 9, 40, 0), ("strided", 1, 0, 6, 5, 2),
+])
+def test_window_grid_and_strided_plans_count_the_oracles_pairs(kind, a, b, gh, gw, T):
+    from oracle import clear_oracle_windows as win
+    okind = win.WINDOWS if kind == "windows" else win.STRIDED
+    ckind = clear.MASK_WINDOWS if kind == "windows" else clear.MASK_STRIDED
+    p = clear.Plan(1, 24, gh, gw, T, 128, a, host_only=True, mask_kind=ckind, mask_param=b)
+    info = p.info()
+    assert info.kernel == clear.KERNEL_SIMT          # no window around the query: the CUDA-core kernel
+    assert info.sum_mask == win.mask_counts(okind, a, b, gh, gw, T)[0]
+    assert info.flops == 4.0 * info.sum_mask * 128 * 24
+
+
+def test_comparison_masks_reproduce_the_papers_flop_figure():
+    # Tab. 1 prints 67.7 GFLOPS for both the Swin-window and the strided baseline at 1024 x 1024 (64 x 64 tokens
+    # + 512 text tokens, c = 3072): 4 * sum(M) * c through the plan
+    for kind, a in ((clear.MASK_WINDOWS, 16), (clear.MASK_STRIDED, 4)):
+        info = clear.Plan(1, 24, 64, 64, 512, 128, a, host_only=True, mask_kind=kind).info()
+        assert round(info.flops / 1e9, 1) in (67.6, 67.7)
+
+
+def test_comparison_mask_plans_reject_bad_arguments():
+    import ctypes
+
+    def rc(kind, size, param, dtype=clear.BF16, d=128):
+        h = ctypes.c_void_p()
+        out = clear.load().clear_plan_create_mask(ctypes.byref(h), 1, 1, 8, 8, 2, d, dtype, kind, size, param, 1)
+        if out == 0:
+            clear.load().clear_plan_destroy(h)
+        return out
+    assert rc(clear.MASK_WINDOWS, 4.0, 1) == 0 and rc(clear.MASK_STRIDED, 3.0, 7, clear.F32, 40) == 0
+    assert rc(clear.MASK_DISC, 4.0, 0) == 0
+    assert rc(clear.MASK_WINDOWS, 4.5, 0) == clear.ERR_INVALID_ARG     # a window is a whole number of cells
+    assert rc(clear.MASK_STRIDED, 0.5, 0) == clear.ERR_INVALID_ARG
+    assert rc(clear.MASK_WINDOWS, 4.0, -1) == clear.ERR_INVALID_ARG
+    assert rc(clear.MASK_DISC, 4.0, 3) == clear.ERR_INVALID_ARG        # the disc takes no second parameter
+    assert rc(7, 4.0, 0) == clear.ERR_INVALID_ARG
+    # the tensor-core kernels' tables do not carry these masks
+    with pytest.raises(clear.ClearError):
+        clear.Plan(1, 1, 8, 8, 2, 128, 4, kernel=clear.KERNEL_TCGEN05_WS, host_only=True, mask_kind=clear.MASK_WINDOWS)
