@@ -170,9 +170,12 @@ int clear_attn_fwd_f32(const void *q, const void *k, const void *v, void *out, i
  *     dS_ij = p_ij (d_out_i . v_j - sum_j' p_ij' d_out_i . v_j'),
  *     dq_i = scale sum_j dS_ij k_j,   dk_j = scale sum_i dS_ij q_i,   dv_j = sum_i p_ij d_out_i.
  * All seven tensors are device pointers, [B, H, N, head_dim] contiguous fp32, 16-byte aligned; q, k, v,
- * d_out are read, dq, dk, dv fully written (dk and dv are zeroed on `stream` first; sums into them are
- * atomic, so their last bits depend on the order of arrival).  Nothing but `stream` is synchronised.
- * A CUDA-core kernel meant for small problems (two atomic adds per channel of every allowed pair).
+ * d_out are read, dq, dk, dv fully written.  Two CUDA-core kernels: one warp per query (row statistics, dq), then
+ * one warp per key (dk, dv; the mask is symmetric, so the queries that see a key are the tokens that key's own
+ * query sees): every output element has one writer and a fixed order of summation, so results repeat bit for
+ * bit.  The first call for a shape allocates 12 bytes per token and (b, h) for the row statistics; calls for one
+ * shape are ordered on the device like those of clear_attn_fwd.  Nothing but `stream` is synchronised.  Meant for
+ * small problems (four dot products per allowed pair on the CUDA cores).
  * Errors: INVALID_ARG, MISALIGNED, UNSUPPORTED (head_dim > 256), CUDA. */
 int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk,
                        void *dv, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius,

@@ -52,6 +52,7 @@ int free_device_parts(clear_plan *p)
     rel(p->d_status);
     rel(p->d_partial_o);
     rel(p->d_partial_ml);
+    rel(p->d_bwd_stats);
     if (p->ev_last) {
         (void)cudaEventDestroy(p->ev_last);
         p->ev_last = nullptr;
@@ -69,6 +70,7 @@ int free_device_parts(clear_plan *p)
     p->d_status = nullptr;
     p->d_partial_o = nullptr;
     p->d_partial_ml = nullptr;
+    p->d_bwd_stats = nullptr;
     return rc;
 }
 
@@ -358,8 +360,17 @@ int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *
     rc = check_tensors(q, k, v, d_out);
     if (rc == CLEAR_OK) rc = check_tensors(dq, dk, dv, dq);
     if (rc != CLEAR_OK) return rc;
-    return with_cached_plan(s, [&](clear_plan_t *plan) {
-        return launch_bwd_f32(*plan, q, k, v, d_out, dq, dk, dv, scale, static_cast<cudaStream_t>(stream));
+    return with_cached_plan(s, [&](clear_plan_t *plan) -> int {
+        // calls of one plan share its row-statistics buffer: ordered on the device like the forward launches
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        std::lock_guard<std::mutex> lock(plan->launch_mutex);
+        if (plan->has_last && plan->last_stream != st) CLEAR_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_last, 0));
+        const int rc2 = launch_bwd_f32(*plan, q, k, v, d_out, dq, dk, dv, scale, st);
+        if (rc2 != CLEAR_OK) return rc2;
+        CLEAR_CUDA_TRY(cudaEventRecord(plan->ev_last, st));
+        plan->last_stream = st;
+        plan->has_last = true;
+        return CLEAR_OK;
     });
 }
 

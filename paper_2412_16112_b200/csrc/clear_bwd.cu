@@ -2,12 +2,15 @@
 // upstream gradient dO of  O = softmax(scale Q K^T + log M) V  (Eq. 1 under the mask of Eq. 3), the step
 // through which the distillation losses of Sec. 3.3 (Eq. 4-6) reach the attention parameters.
 //
-// One warp per query, lanes split the head dimension, keys walked as in the forward CUDA-core kernel (the
-// text tokens, then per grid row within reach the clipped run of columns).  Two sweeps over the allowed keys:
-//   1. online softmax: row maximum m, row sum l, the un-normalised output, hence delta = dO . O;
-//   2. per key: p = exp(s - m) / l, dP = dO . v, dS = p (dP - delta);  dQ += scale dS k  (registers),
-//      dK_j += scale dS q  and  dV_j += p dO  (atomic adds: several queries share a key).
-// Sized for small problems (the fp32 configuration): 2 d atomic adds per allowed pair.
+// Two kernels, one warp per token, lanes split the head dimension, tokens walked as in the forward CUDA-core
+// kernel (the text tokens, then per grid row within reach the clipped run of columns):
+//   query kernel: sweep 1 over the query's keys: online softmax -> row maximum m, row sum l, the un-normalised
+//       output, hence delta = dO . O; the three row statistics are kept for the second kernel;
+//       sweep 2: p = exp(s - m) / l, dP = dO . v, dS = p (dP - delta), dQ += scale dS k;
+//   key kernel: the mask is symmetric (M_ij = M_ji), so the queries that see key j are the tokens query j sees:
+//       for each of them p_ij and dS_ij again from that query's statistics, dK_j += scale dS q_i, dV_j += p dO_i.
+// Every output element has one writer and a fixed order of summation: results are the same from run to run.
+// Each allowed pair costs four dot products of d channels instead of two, and no atomic operation.
 #include "clear_internal.hpp"
 
 namespace clear {
@@ -24,9 +27,9 @@ __device__ __forceinline__ float warp_sum(float x)
 
 template <int EPL>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
-clear_bwd_kernel(const float *__restrict__ q, const float *__restrict__ k, const float *__restrict__ v,
-                 const float *__restrict__ d_out, float *__restrict__ dq, float *dk, float *dv, int grid_h, int grid_w,
-                 int n_text, int d, const int32_t *__restrict__ half_width, int n_half_width, float scale)
+clear_bwd_query_kernel(const float *__restrict__ q, const float *__restrict__ k, const float *__restrict__ v,
+                       const float *__restrict__ d_out, float *__restrict__ dq, float *__restrict__ stats, int grid_h,
+                       int grid_w, int n_text, int d, const int32_t *__restrict__ half_width, int n_half_width, float scale)
 {
     const int lane = threadIdx.x & 31;
     const int64_t N = (int64_t)n_text + (int64_t)grid_h * grid_w;
@@ -93,6 +96,12 @@ clear_bwd_kernel(const float *__restrict__ q, const float *__restrict__ k, const
 #pragma unroll
     for (int t = 0; t < EPL; ++t) part = fmaf(gv[t], acc[t], part);
     const float delta = warp_sum(part) * inv_l;  // dO . O = sum_j p_ij dP_ij
+    if (lane == 0) {
+        float *st = stats + ((int64_t)blockIdx.y * N + i) * 3;
+        st[0] = m;
+        st[1] = inv_l;
+        st[2] = delta;
+    }
 
     // ---- sweep 2: the gradients --------------------------------------------------------------------
     float gq[EPL];
@@ -105,11 +114,7 @@ clear_bwd_kernel(const float *__restrict__ q, const float *__restrict__ k, const
 #pragma unroll
             for (int t = 0; t < EPL; ++t) {
                 const int e = lane + 32 * t;
-                if (e < d) {
-                    gq[t] = fmaf(ds, k[base + j * d + e], gq[t]);
-                    atomicAdd(dk + base + j * d + e, ds * qv[t]);
-                    atomicAdd(dv + base + j * d + e, p * gv[t]);
-                }
+                if (e < d) gq[t] = fmaf(ds, k[base + j * d + e], gq[t]);
             }
         }
     });
@@ -120,6 +125,79 @@ clear_bwd_kernel(const float *__restrict__ q, const float *__restrict__ k, const
     }
 }
 
+// dK_j, dV_j: one warp per key j; the tokens that see key j are the tokens query j sees (symmetric mask).
+template <int EPL>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+clear_bwd_key_kernel(const float *__restrict__ q, const float *__restrict__ k, const float *__restrict__ v,
+                     const float *__restrict__ d_out, const float *__restrict__ stats, float *__restrict__ dk,
+                     float *__restrict__ dv, int grid_h, int grid_w, int n_text, int d,
+                     const int32_t *__restrict__ half_width, int n_half_width, float scale)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t N = (int64_t)n_text + (int64_t)grid_h * grid_w;
+    const int64_t j = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (j >= N) return;  // whole warp leaves together
+    const int64_t base = (int64_t)blockIdx.y * N * d;
+    const float *st = stats + (int64_t)blockIdx.y * N * 3;
+
+    float kv[EPL], vv[EPL], gk[EPL], gv[EPL];
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) {
+        const int e = lane + 32 * t;
+        kv[t] = e < d ? k[base + j * d + e] : 0.f;
+        vv[t] = e < d ? v[base + j * d + e] : 0.f;
+        gk[t] = gv[t] = 0.f;
+    }
+    auto dot_row = [&](const float (&a)[EPL], const float *__restrict__ rows, int64_t i) {
+        float part = 0.f;
+#pragma unroll
+        for (int t = 0; t < EPL; ++t) {
+            const int e = lane + 32 * t;
+            if (e < d) part = fmaf(a[t], rows[base + i * d + e], part);
+        }
+        return warp_sum(part);
+    };
+    auto run = [&](int64_t i0, int64_t i1) {
+        for (int64_t i = i0; i < i1; ++i) {
+            const float m = st[i * 3], inv_l = st[i * 3 + 1], delta = st[i * 3 + 2];
+            const float p = expf(scale * dot_row(kv, q, i) - m) * inv_l;
+            const float ds = p * (dot_row(vv, d_out, i) - delta) * scale;
+#pragma unroll
+            for (int t = 0; t < EPL; ++t) {
+                const int e = lane + 32 * t;
+                if (e < d) {
+                    gk[t] = fmaf(ds, q[base + i * d + e], gk[t]);
+                    gv[t] = fmaf(p, d_out[base + i * d + e], gv[t]);
+                }
+            }
+        }
+    };
+    if (j < n_text) {
+        run(0, N);  // every query sees a text key
+    } else {
+        run(0, n_text);  // every text query sees every image key
+        const int64_t pix = j - n_text;
+        const int y = (int)(pix / grid_w), x = (int)(pix % grid_w);
+        const int R = n_half_width - 1;
+        for (int dy = -R; dy <= R; ++dy) {
+            const int yy = y + dy;
+            if (yy < 0 || yy >= grid_h) continue;
+            const int hw = half_width[dy < 0 ? -dy : dy];
+            const int lo = max(x - hw, 0), hi = min(x + hw, grid_w - 1);
+            const int64_t row0 = (int64_t)n_text + (int64_t)yy * grid_w;
+            run(row0 + lo, row0 + hi + 1);
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < EPL; ++t) {
+        const int e = lane + 32 * t;
+        if (e < d) {
+            dk[base + j * d + e] = gk[t];
+            dv[base + j * d + e] = gv[t];
+        }
+    }
+}
+
 }  // namespace
 
 int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq,
@@ -127,20 +205,29 @@ int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void
 {
     const Shape &s = p.shape;
     const int64_t N = (int64_t)s.n_text + (int64_t)s.grid_h * s.grid_w;
-    const size_t bytes = (size_t)s.B * s.H * N * s.head_dim * sizeof(float);
-    // several queries add into one key's gradients: they start at zero
-    CLEAR_CUDA_TRY(cudaMemsetAsync(dk, 0, bytes, stream));
-    CLEAR_CUDA_TRY(cudaMemsetAsync(dv, 0, bytes, stream));
+    // row statistics (m, 1 / l, delta) of every query: owned by the plan, allocated on its first backward call
+    // (calls of one plan are ordered on the device, so one buffer serves them all)
+    if (!p.d_bwd_stats) {
+        cudaError_t e = cudaMalloc((void **)&p.d_bwd_stats, (size_t)s.B * s.H * N * 3 * sizeof(float));
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            return e == cudaErrorMemoryAllocation ? CLEAR_ERR_NO_MEMORY : CLEAR_ERR_CUDA;
+        }
+    }
     dim3 grid((unsigned)((N + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)(s.B * s.H));
     dim3 block(kWarpsPerBlock * 32);
     const int n_hw = (int)p.sch.half_width.size();
     const int epl = (s.head_dim + 31) / 32;
-#define CLEAR_BWD_CASE(E)                                                                                            \
-    case E:                                                                                                          \
-        clear_bwd_kernel<E><<<grid, block, 0, stream>>>((const float *)q, (const float *)k, (const float *)v,       \
-                                                        (const float *)d_out, (float *)dq, (float *)dk, (float *)dv, \
-                                                        s.grid_h, s.grid_w, s.n_text, s.head_dim, p.d_half_width,    \
-                                                        n_hw, scale);                                                \
+#define CLEAR_BWD_CASE(E)                                                                                               \
+    case E:                                                                                                             \
+        clear_bwd_query_kernel<E><<<grid, block, 0, stream>>>((const float *)q, (const float *)k, (const float *)v,    \
+                                                              (const float *)d_out, (float *)dq, p.d_bwd_stats,         \
+                                                              s.grid_h, s.grid_w, s.n_text, s.head_dim,                 \
+                                                              p.d_half_width, n_hw, scale);                             \
+        clear_bwd_key_kernel<E><<<grid, block, 0, stream>>>((const float *)q, (const float *)k, (const float *)v,      \
+                                                            (const float *)d_out, p.d_bwd_stats, (float *)dk,           \
+                                                            (float *)dv, s.grid_h, s.grid_w, s.n_text, s.head_dim,      \
+                                                            p.d_half_width, n_hw, scale);                               \
         break;
     switch (epl) {
         CLEAR_BWD_CASE(1)

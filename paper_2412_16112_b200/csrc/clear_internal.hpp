@@ -60,6 +60,8 @@ struct clear_plan {
     // un-normalised outputs, and per row the running maximum (log2 units) and the row sum
     float *d_partial_o = nullptr;
     float *d_partial_ml = nullptr;
+    // backward pass: (m, 1 / l, delta) per query row, allocated on the plan's first backward call
+    mutable float *d_bwd_stats = nullptr;
     int64_t workspace_bytes = 0;
 
     // staging buffers of the host-tensor entry point (owned, allocated on first use)

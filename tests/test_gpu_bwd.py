@@ -53,3 +53,33 @@ def test_backward_argument_errors():
     assert lib.clear_attn_bwd_f32(p, p, p, None, p, p, p, 1, 1, 16, 16, 16, 64, 4.0, 0.125, None) == clear.ERR_INVALID_ARG
     assert lib.clear_attn_bwd_f32(p, p, p, p, p, p + 4, p, 1, 1, 16, 16, 16, 64, 4.0, 0.125, None) == clear.ERR_MISALIGNED
     assert lib.clear_attn_bwd_f32(p, p, p, p, p, p, p, 1, 1, 16, 16, 16, 64, 4.0, float("nan"), None) == clear.ERR_INVALID_ARG
+
+
+def test_backward_repeats_bit_for_bit_and_from_two_streams():
+    """One writer per output element and a fixed order of summation: the same bits on every call, also when two
+    streams call for the same shape at once (the library orders them: they share the row statistics)."""
+    gh, gw, T, r, d = 24, 40, 130, 8.0, 64
+    q, k, v = workloads.make_custom(1, 3, gh, gw, T, d, dtype="f32", qk_norm=False, seed=5)
+    g = torch.Generator(device="cpu").manual_seed(6)
+    d_out = torch.randn(q.shape, generator=g, dtype=torch.float32)
+    scale = 1 / math.sqrt(d)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, gd = (t.to(dev) for t in (q, k, v, d_out))
+    first = [torch.full_like(qd, float("nan")) for _ in range(3)]
+    clear.clear_attn_bwd_f32(qd, kd, vd, gd, *first, gh, gw, T, r, scale)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    # the second stream gets other inputs, so a mix-up of the shared statistics would show
+    q2 = (qd * 1.5).contiguous()
+    outs = [[torch.full_like(qd, float("nan")) for _ in range(3)] for _ in range(2)]
+    for rep in range(3):
+        for s, (qq, o) in zip(streams, ((qd, outs[0]), (q2, outs[1]))):
+            with torch.cuda.stream(s):
+                clear.clear_attn_bwd_f32(qq, kd, vd, gd, *o, gh, gw, T, r, scale, stream=s)
+    torch.cuda.synchronize()
+    for a, b in zip(first, outs[0]):
+        assert torch.equal(a, b)
+    want = oracle_bwd.attn_bwd(q * 1.5, k, v, d_out, gh, gw, T, r, scale)
+    for got, ref in zip(outs[1], want):
+        assert np.abs(got.cpu().double().numpy() - ref).max() <= BWD_ATOL
+    clear.clear_cache_clear()
