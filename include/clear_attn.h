@@ -181,6 +181,12 @@ int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *
                        void *dv, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius,
                        float scale, void *stream);
 
+/* The same backward pass for bf16 tensors (all seven; 16-byte aligned): fp32 arithmetic and statistics as above,
+ * gradients rounded to bf16 (nearest even) when stored.  Same kernels, errors and stream rules. */
+int clear_attn_bwd_bf16(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk,
+                        void *dv, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius,
+                        float scale, void *stream);
+
 /* What the model does to Q and K between their projections and the attention call, in one pass over memory:
  * RMS normalisation over the head's channels, rotary position embedding on the two axes of the feature map
  * (Sec. 3.1: the model perceives spatial relations through it, by the relative distances on the two axes), with

@@ -33,7 +33,7 @@ EXPORTS = [
     "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim", "clear_attn_bwd_f32", "clear_plan_create_ex",
     "clear_qk_norm_rope", "clear_log_scale_factor",
     "clear_band_geometry", "clear_plan_create_band", "clear_attn_text_partial", "clear_text_merge",
-    "clear_plan_create_mask",
+    "clear_plan_create_mask", "clear_attn_bwd_bf16",
 ]
 
 
@@ -97,6 +97,7 @@ def load() -> ctypes.CDLL:
         lib.clear_attn_fwd_f32.argtypes = fwd_args
         lib.clear_attn_fwd_static.argtypes = fwd_args
         lib.clear_attn_bwd_f32.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp]
+        lib.clear_attn_bwd_bf16.argtypes = lib.clear_attn_bwd_f32.argtypes
         lib.clear_qk_norm_rope.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, i32,
                                            f32, f32, f32, f32, vp]
         pi32 = ctypes.POINTER(ctypes.c_int32)
@@ -190,17 +191,29 @@ def clear_attn_fwd(q, k, v, out, grid_h, grid_w, n_text, radius, scale, stream=N
     return out
 
 
+def _backward(fn_name, dtype, q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radius, scale, stream):
+    for t in (q, k, v, d_out, dq, dk, dv):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype and t.shape == q.shape):
+            raise ValueError(f"backward tensors must be contiguous {dtype} CUDA tensors of one [B, H, N, d] shape")
+    B, H, _, d = q.shape
+    _check(getattr(load(), fn_name)(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_out.data_ptr(), dq.data_ptr(),
+                                    dk.data_ptr(), dv.data_ptr(), B, H, grid_h, grid_w, n_text, d, float(radius),
+                                    float(scale), _stream_ptr(stream)), fn_name)
+    return dq, dk, dv
+
+
 def clear_attn_bwd_f32(q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radius, scale, stream=None):
     """fp32 backward pass: gradients of q, k, v into ``dq``, ``dk``, ``dv`` for the upstream gradient ``d_out``."""
     import torch
-    for t in (q, k, v, d_out, dq, dk, dv):
-        if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.float32 and t.shape == q.shape):
-            raise ValueError("backward tensors must be contiguous fp32 CUDA tensors of one [B, H, N, d] shape")
-    B, H, _, d = q.shape
-    _check(load().clear_attn_bwd_f32(q.data_ptr(), k.data_ptr(), v.data_ptr(), d_out.data_ptr(), dq.data_ptr(),
-                                     dk.data_ptr(), dv.data_ptr(), B, H, grid_h, grid_w, n_text, d, float(radius),
-                                     float(scale), _stream_ptr(stream)), "clear_attn_bwd_f32")
-    return dq, dk, dv
+    return _backward("clear_attn_bwd_f32", torch.float32, q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radius,
+                     scale, stream)
+
+
+def clear_attn_bwd_bf16(q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radius, scale, stream=None):
+    """The same for bf16 tensors (fp32 arithmetic, gradients rounded to bf16)."""
+    import torch
+    return _backward("clear_attn_bwd_bf16", torch.bfloat16, q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radius,
+                     scale, stream)
 
 
 def clear_qk_norm_rope(q, k, q_out, k_out, grid_h, grid_w, n_text, axes_dim, gain_q=None, gain_k=None, theta=10000.0,

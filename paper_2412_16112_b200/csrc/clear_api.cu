@@ -349,11 +349,11 @@ int clear_attn_fwd_f32(const void *q, const void *k, const void *v, void *out, i
     return cached_forward(q, k, v, out, s, scale, stream);
 }
 
-int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk, void *dv,
-                       int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale,
-                       void *stream)
+static int backward(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk, void *dv, int B,
+                    int H, int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale, int dtype,
+                    void *stream)
 {
-    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, CLEAR_F32, CLEAR_KERNEL_SIMT};
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, dtype, CLEAR_KERNEL_SIMT};
     int rc = validate_shape(s);
     if (rc != CLEAR_OK) return rc;
     if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
@@ -365,13 +365,27 @@ int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *
         cudaStream_t st = static_cast<cudaStream_t>(stream);
         std::lock_guard<std::mutex> lock(plan->launch_mutex);
         if (plan->has_last && plan->last_stream != st) CLEAR_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_last, 0));
-        const int rc2 = launch_bwd_f32(*plan, q, k, v, d_out, dq, dk, dv, scale, st);
+        const int rc2 = launch_bwd(*plan, q, k, v, d_out, dq, dk, dv, scale, st);
         if (rc2 != CLEAR_OK) return rc2;
         CLEAR_CUDA_TRY(cudaEventRecord(plan->ev_last, st));
         plan->last_stream = st;
         plan->has_last = true;
         return CLEAR_OK;
     });
+}
+
+int clear_attn_bwd_f32(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk, void *dv,
+                       int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale,
+                       void *stream)
+{
+    return backward(q, k, v, d_out, dq, dk, dv, B, H, grid_h, grid_w, n_text, head_dim, radius, scale, CLEAR_F32, stream);
+}
+
+int clear_attn_bwd_bf16(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk, void *dv,
+                        int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale,
+                        void *stream)
+{
+    return backward(q, k, v, d_out, dq, dk, dv, B, H, grid_h, grid_w, n_text, head_dim, radius, scale, CLEAR_BF16, stream);
 }
 
 int clear_qk_norm_rope(const void *q_in, const void *k_in, void *q_out, void *k_out, const float *gain_q,

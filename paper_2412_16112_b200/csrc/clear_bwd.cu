@@ -11,12 +11,19 @@
 //       for each of them p_ij and dS_ij again from that query's statistics, dK_j += scale dS q_i, dV_j += p dO_i.
 // Every output element has one writer and a fixed order of summation: results are the same from run to run.
 // Each allowed pair costs four dot products of d channels instead of two, and no atomic operation.
+#include <cuda_bf16.h>
+
 #include "clear_internal.hpp"
 
 namespace clear {
 namespace {
 
 constexpr int kWarpsPerBlock = 8;
+
+__device__ __forceinline__ float ldf(const float *p) { return *p; }
+__device__ __forceinline__ float ldf(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void stf(float *p, float x) { *p = x; }
+__device__ __forceinline__ void stf(__nv_bfloat16 *p, float x) { *p = __float2bfloat16_rn(x); }
 
 __device__ __forceinline__ float warp_sum(float x)
 {
@@ -25,10 +32,10 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
-template <int EPL>
+template <typename T, int EPL>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
-clear_bwd_query_kernel(const float *__restrict__ q, const float *__restrict__ k, const float *__restrict__ v,
-                       const float *__restrict__ d_out, float *__restrict__ dq, float *__restrict__ stats, int grid_h,
+clear_bwd_query_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
+                       const T *__restrict__ d_out, T *__restrict__ dq, float *__restrict__ stats, int grid_h,
                        int grid_w, int n_text, int d, const int32_t *__restrict__ half_width, int n_half_width, float scale)
 {
     const int lane = threadIdx.x & 31;
@@ -41,16 +48,16 @@ clear_bwd_query_kernel(const float *__restrict__ q, const float *__restrict__ k,
 #pragma unroll
     for (int t = 0; t < EPL; ++t) {
         const int e = lane + 32 * t;
-        qv[t] = e < d ? q[base + i * d + e] : 0.f;
-        gv[t] = e < d ? d_out[base + i * d + e] : 0.f;
+        qv[t] = e < d ? ldf(q + base + i * d + e) : 0.f;
+        gv[t] = e < d ? ldf(d_out + base + i * d + e) : 0.f;
         acc[t] = 0.f;
     }
-    auto dot_row = [&](const float (&a)[EPL], const float *__restrict__ rows, int64_t j) {
+    auto dot_row = [&](const float (&a)[EPL], const T *__restrict__ rows, int64_t j) {
         float part = 0.f;
 #pragma unroll
         for (int t = 0; t < EPL; ++t) {
             const int e = lane + 32 * t;
-            if (e < d) part = fmaf(a[t], rows[base + j * d + e], part);
+            if (e < d) part = fmaf(a[t], ldf(rows + base + j * d + e), part);
         }
         return warp_sum(part);
     };
@@ -86,7 +93,7 @@ clear_bwd_query_kernel(const float *__restrict__ q, const float *__restrict__ k,
 #pragma unroll
             for (int t = 0; t < EPL; ++t) {
                 const int e = lane + 32 * t;
-                if (e < d) acc[t] = fmaf(p, v[base + j * d + e], acc[t] * alpha);
+                if (e < d) acc[t] = fmaf(p, ldf(v + base + j * d + e), acc[t] * alpha);
             }
             m = m_new;
         }
@@ -114,23 +121,23 @@ clear_bwd_query_kernel(const float *__restrict__ q, const float *__restrict__ k,
 #pragma unroll
             for (int t = 0; t < EPL; ++t) {
                 const int e = lane + 32 * t;
-                if (e < d) gq[t] = fmaf(ds, k[base + j * d + e], gq[t]);
+                if (e < d) gq[t] = fmaf(ds, ldf(k + base + j * d + e), gq[t]);
             }
         }
     });
 #pragma unroll
     for (int t = 0; t < EPL; ++t) {
         const int e = lane + 32 * t;
-        if (e < d) dq[base + i * d + e] = gq[t];
+        if (e < d) stf(dq + base + i * d + e, gq[t]);
     }
 }
 
 // dK_j, dV_j: one warp per key j; the tokens that see key j are the tokens query j sees (symmetric mask).
-template <int EPL>
+template <typename T, int EPL>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
-clear_bwd_key_kernel(const float *__restrict__ q, const float *__restrict__ k, const float *__restrict__ v,
-                     const float *__restrict__ d_out, const float *__restrict__ stats, float *__restrict__ dk,
-                     float *__restrict__ dv, int grid_h, int grid_w, int n_text, int d,
+clear_bwd_key_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
+                     const T *__restrict__ d_out, const float *__restrict__ stats, T *__restrict__ dk,
+                     T *__restrict__ dv, int grid_h, int grid_w, int n_text, int d,
                      const int32_t *__restrict__ half_width, int n_half_width, float scale)
 {
     const int lane = threadIdx.x & 31;
@@ -144,16 +151,16 @@ clear_bwd_key_kernel(const float *__restrict__ q, const float *__restrict__ k, c
 #pragma unroll
     for (int t = 0; t < EPL; ++t) {
         const int e = lane + 32 * t;
-        kv[t] = e < d ? k[base + j * d + e] : 0.f;
-        vv[t] = e < d ? v[base + j * d + e] : 0.f;
+        kv[t] = e < d ? ldf(k + base + j * d + e) : 0.f;
+        vv[t] = e < d ? ldf(v + base + j * d + e) : 0.f;
         gk[t] = gv[t] = 0.f;
     }
-    auto dot_row = [&](const float (&a)[EPL], const float *__restrict__ rows, int64_t i) {
+    auto dot_row = [&](const float (&a)[EPL], const T *__restrict__ rows, int64_t i) {
         float part = 0.f;
 #pragma unroll
         for (int t = 0; t < EPL; ++t) {
             const int e = lane + 32 * t;
-            if (e < d) part = fmaf(a[t], rows[base + i * d + e], part);
+            if (e < d) part = fmaf(a[t], ldf(rows + base + i * d + e), part);
         }
         return warp_sum(part);
     };
@@ -166,8 +173,8 @@ clear_bwd_key_kernel(const float *__restrict__ q, const float *__restrict__ k, c
             for (int t = 0; t < EPL; ++t) {
                 const int e = lane + 32 * t;
                 if (e < d) {
-                    gk[t] = fmaf(ds, q[base + i * d + e], gk[t]);
-                    gv[t] = fmaf(p, d_out[base + i * d + e], gv[t]);
+                    gk[t] = fmaf(ds, ldf(q + base + i * d + e), gk[t]);
+                    gv[t] = fmaf(p, ldf(d_out + base + i * d + e), gv[t]);
                 }
             }
         }
@@ -192,16 +199,15 @@ clear_bwd_key_kernel(const float *__restrict__ q, const float *__restrict__ k, c
     for (int t = 0; t < EPL; ++t) {
         const int e = lane + 32 * t;
         if (e < d) {
-            dk[base + j * d + e] = gk[t];
-            dv[base + j * d + e] = gv[t];
+            stf(dk + base + j * d + e, gk[t]);
+            stf(dv + base + j * d + e, gv[t]);
         }
     }
 }
 
-}  // namespace
-
-int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq,
-                   void *dk, void *dv, float scale, cudaStream_t stream)
+template <typename T>
+int launch_bwd_typed(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq,
+                     void *dk, void *dv, float scale, cudaStream_t stream)
 {
     const Shape &s = p.shape;
     const int64_t N = (int64_t)s.n_text + (int64_t)s.grid_h * s.grid_w;
@@ -220,14 +226,14 @@ int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void
     const int epl = (s.head_dim + 31) / 32;
 #define CLEAR_BWD_CASE(E)                                                                                               \
     case E:                                                                                                             \
-        clear_bwd_query_kernel<E><<<grid, block, 0, stream>>>((const float *)q, (const float *)k, (const float *)v,    \
-                                                              (const float *)d_out, (float *)dq, p.d_bwd_stats,         \
-                                                              s.grid_h, s.grid_w, s.n_text, s.head_dim,                 \
-                                                              p.d_half_width, n_hw, scale);                             \
-        clear_bwd_key_kernel<E><<<grid, block, 0, stream>>>((const float *)q, (const float *)k, (const float *)v,      \
-                                                            (const float *)d_out, p.d_bwd_stats, (float *)dk,           \
-                                                            (float *)dv, s.grid_h, s.grid_w, s.n_text, s.head_dim,      \
-                                                            p.d_half_width, n_hw, scale);                               \
+        clear_bwd_query_kernel<T, E><<<grid, block, 0, stream>>>((const T *)q, (const T *)k, (const T *)v,             \
+                                                                 (const T *)d_out, (T *)dq, p.d_bwd_stats, s.grid_h,    \
+                                                                 s.grid_w, s.n_text, s.head_dim, p.d_half_width, n_hw,  \
+                                                                 scale);                                                \
+        clear_bwd_key_kernel<T, E><<<grid, block, 0, stream>>>((const T *)q, (const T *)k, (const T *)v,               \
+                                                               (const T *)d_out, p.d_bwd_stats, (T *)dk, (T *)dv,       \
+                                                               s.grid_h, s.grid_w, s.n_text, s.head_dim,                \
+                                                               p.d_half_width, n_hw, scale);                            \
         break;
     switch (epl) {
         CLEAR_BWD_CASE(1)
@@ -244,6 +250,15 @@ int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void
 #undef CLEAR_BWD_CASE
     CLEAR_CUDA_TRY(cudaGetLastError());
     return CLEAR_OK;
+}
+
+}  // namespace
+
+int launch_bwd(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk,
+               void *dv, float scale, cudaStream_t stream)
+{
+    if (p.shape.dtype == CLEAR_F32) return launch_bwd_typed<float>(p, q, k, v, d_out, dq, dk, dv, scale, stream);
+    return launch_bwd_typed<__nv_bfloat16>(p, q, k, v, d_out, dq, dk, dv, scale, stream);
 }
 
 }  // namespace clear

@@ -99,9 +99,9 @@ int launch_tc(const clear_plan &p, const void *q, const void *k, const void *v, 
               cudaStream_t stream);
 int launch_ws(const clear_plan &p, const void *q, const void *k, const void *v, void *out, float scale,
               cudaStream_t stream);
-// fp32 backward pass on the CUDA cores (dk and dv are zeroed on the stream first).
-int launch_bwd_f32(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq,
-                   void *dk, void *dv, float scale, cudaStream_t stream);
+// Backward pass on the CUDA cores (fp32 arithmetic; tensors of the plan's dtype): a query kernel and a key kernel.
+int launch_bwd(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk,
+               void *dv, float scale, cudaStream_t stream);
 // Row-band form: one (O, m, l) record per text row from a band-text plan's partial results, and the merge of the
 // records of all bands into bf16 text rows.
 int launch_text_export(const clear_plan &p, void *records, cudaStream_t stream);

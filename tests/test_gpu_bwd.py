@@ -83,3 +83,24 @@ def test_backward_repeats_bit_for_bit_and_from_two_streams():
     for got, ref in zip(outs[1], want):
         assert np.abs(got.cpu().double().numpy() - ref).max() <= BWD_ATOL
     clear.clear_cache_clear()
+
+
+@pytest.mark.parametrize("gh,gw,T,r,d", [(16, 24, 20, 4.0, 128), (13, 19, 7, 2.5, 64), (24, 40, 130, 8.0, 128)])
+def test_bf16_backward_matches_the_oracle(gh, gw, T, r, d):
+    """bf16 tensors in and out, fp32 arithmetic: the error is the rounding of each gradient to bf16 (half a unit
+    in the last of 8 significant bits) on top of the fp32 kernel's."""
+    q, k, v = workloads.make_custom(1, 2, gh, gw, T, d, dtype="bf16", seed=gh + gw)
+    g = torch.Generator(device="cpu").manual_seed(gh * gw)
+    d_out = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16)
+    scale = 1 / math.sqrt(d)
+    want = oracle_bwd.attn_bwd(q, k, v, d_out, gh, gw, T, r, scale)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, gd = (t.to(dev) for t in (q, k, v, d_out))
+    dq, dk, dv = (torch.full_like(qd, float("nan")) for _ in range(3))
+    clear.clear_attn_bwd_bf16(qd, kd, vd, gd, dq, dk, dv, gh, gw, T, r, scale)
+    torch.cuda.synchronize()
+    for name, got, ref in (("dq", dq, want[0]), ("dk", dk, want[1]), ("dv", dv, want[2])):
+        err = np.abs(got.cpu().double().numpy() - ref)
+        assert np.isfinite(err).all(), f"{name}: non-finite"
+        assert (err <= 2.0 ** -8 * np.abs(ref) + BWD_ATOL).all(), f"{name}: max {err.max():.3e}"
+    clear.clear_cache_clear()
