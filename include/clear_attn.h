@@ -217,6 +217,19 @@ int clear_qk_norm_rope(const void *q_in, const void *k_in, void *q_out, void *k_
  * beyond the training resolution).  Host arithmetic only; 1 when either count is below 2. */
 float clear_log_scale_factor(long long n_tokens, long long n_train_tokens);
 
+/* The backward pass for bf16 tensors on the tensor cores (head_dim 64 or 128, scale > 0): same arguments and
+ * results as clear_attn_bwd_bf16, computed with tcgen05 MMAs over the forward pass's tile schedule -- a launch in
+ * which every 128-query tile meets its key tiles (row statistics and delta = dO . O in a first sweep, dQ in a second)
+ * and a launch in which every 128-key tile meets the query tiles that see it (dK, dV; Eq. 3's mask is symmetric, so
+ * these are the same lists).  P and dS enter the MMAs rounded to bf16, as P does in the forward pass: gradients
+ * agree with the exact ones to about 1e-2 of the largest gradient of the tensor.  One writer per element: results
+ * repeat bit for bit.  The first call for a shape allocates its schedule tables and 16 bytes per token and (b, h).
+ * Errors: INVALID_ARG, MISALIGNED, UNSUPPORTED (other head sizes, scale <= 0), CUDA; a kernel whose bounded wait
+ * expired is found by clear_cache_check. */
+int clear_attn_bwd_bf16_tc(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk,
+                           void *dv, int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius,
+                           float scale, void *stream);
+
 /* Window of an image query (text tokens are always allowed, as in Eq. 3). */
 enum {
     CLEAR_MASK_DISC = 0,   /* Eq. 3: dx^2 + dy^2 < r^2, the paper's circular window                              */

@@ -33,7 +33,7 @@ EXPORTS = [
     "clear_last_device_status", "clear_plan_mask_table", "clear_cache_check", "clear_plan_trim", "clear_attn_bwd_f32", "clear_plan_create_ex",
     "clear_qk_norm_rope", "clear_log_scale_factor",
     "clear_band_geometry", "clear_plan_create_band", "clear_attn_text_partial", "clear_text_merge",
-    "clear_plan_create_mask", "clear_attn_bwd_bf16",
+    "clear_plan_create_mask", "clear_attn_bwd_bf16", "clear_attn_bwd_bf16_tc",
 ]
 
 
@@ -98,6 +98,7 @@ def load() -> ctypes.CDLL:
         lib.clear_attn_fwd_static.argtypes = fwd_args
         lib.clear_attn_bwd_f32.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp]
         lib.clear_attn_bwd_bf16.argtypes = lib.clear_attn_bwd_f32.argtypes
+        lib.clear_attn_bwd_bf16_tc.argtypes = lib.clear_attn_bwd_f32.argtypes
         lib.clear_qk_norm_rope.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, i32,
                                            f32, f32, f32, f32, vp]
         pi32 = ctypes.POINTER(ctypes.c_int32)
@@ -214,6 +215,13 @@ def clear_attn_bwd_bf16(q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radi
     import torch
     return _backward("clear_attn_bwd_bf16", torch.bfloat16, q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radius,
                      scale, stream)
+
+
+def clear_attn_bwd_bf16_tc(q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text, radius, scale, stream=None):
+    """bf16 backward pass on the tensor cores (head size 64 or 128)."""
+    import torch
+    return _backward("clear_attn_bwd_bf16_tc", torch.bfloat16, q, k, v, d_out, dq, dk, dv, grid_h, grid_w, n_text,
+                     radius, scale, stream)
 
 
 def clear_qk_norm_rope(q, k, q_out, k_out, grid_h, grid_w, n_text, axes_dim, gain_q=None, gain_k=None, theta=10000.0,

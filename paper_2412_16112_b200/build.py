@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB = os.path.join(LIB_DIR, "libclear_attn.so")
-SOURCES = ["clear_api.cu", "clear_plan.cpp", "clear_simt.cu", "clear_tc.cu", "clear_ws.cu", "clear_static.cu", "clear_tma.cu", "clear_bwd.cu", "clear_prep.cu", "clear_bands.cu"]
+SOURCES = ["clear_api.cu", "clear_plan.cpp", "clear_simt.cu", "clear_tc.cu", "clear_ws.cu", "clear_static.cu", "clear_tma.cu", "clear_bwd.cu", "clear_prep.cu", "clear_bands.cu", "clear_bwd_tc.cu"]
 
 
 def _nvcc() -> str:

@@ -351,9 +351,10 @@ int clear_attn_fwd_f32(const void *q, const void *k, const void *v, void *out, i
 
 static int backward(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk, void *dv, int B,
                     int H, int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale, int dtype,
-                    void *stream)
+                    void *stream, bool tensor_cores = false)
 {
-    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, dtype, CLEAR_KERNEL_SIMT};
+    Shape s{B, H, grid_h, grid_w, n_text, head_dim, radius, dtype, tensor_cores ? CLEAR_KERNEL_TCGEN05 : CLEAR_KERNEL_SIMT};
+    s.no_text_split = tensor_cores ? 1 : 0;
     int rc = validate_shape(s);
     if (rc != CLEAR_OK) return rc;
     if (!std::isfinite(scale)) return CLEAR_ERR_INVALID_ARG;
@@ -365,7 +366,8 @@ static int backward(const void *q, const void *k, const void *v, const void *d_o
         cudaStream_t st = static_cast<cudaStream_t>(stream);
         std::lock_guard<std::mutex> lock(plan->launch_mutex);
         if (plan->has_last && plan->last_stream != st) CLEAR_CUDA_TRY(cudaStreamWaitEvent(st, plan->ev_last, 0));
-        const int rc2 = launch_bwd(*plan, q, k, v, d_out, dq, dk, dv, scale, st);
+        const int rc2 = tensor_cores ? launch_bwd_tc(*plan, q, k, v, d_out, dq, dk, dv, scale, st)
+                                     : launch_bwd(*plan, q, k, v, d_out, dq, dk, dv, scale, st);
         if (rc2 != CLEAR_OK) return rc2;
         CLEAR_CUDA_TRY(cudaEventRecord(plan->ev_last, st));
         plan->last_stream = st;
@@ -386,6 +388,16 @@ int clear_attn_bwd_bf16(const void *q, const void *k, const void *v, const void 
                         void *stream)
 {
     return backward(q, k, v, d_out, dq, dk, dv, B, H, grid_h, grid_w, n_text, head_dim, radius, scale, CLEAR_BF16, stream);
+}
+
+int clear_attn_bwd_bf16_tc(const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk, void *dv,
+                           int B, int H, int grid_h, int grid_w, int n_text, int head_dim, float radius, float scale,
+                           void *stream)
+{
+    if (head_dim != 64 && head_dim != 128) return CLEAR_ERR_UNSUPPORTED;
+    if (!(scale > 0.f)) return std::isfinite(scale) ? CLEAR_ERR_UNSUPPORTED : CLEAR_ERR_INVALID_ARG;
+    return backward(q, k, v, d_out, dq, dk, dv, B, H, grid_h, grid_w, n_text, head_dim, radius, scale, CLEAR_BF16, stream,
+                    true);
 }
 
 int clear_qk_norm_rope(const void *q_in, const void *k_in, void *q_out, void *k_out, const float *gain_q,

@@ -111,6 +111,10 @@ int launch_text_merge(const float *records, int n_parts, int n_bh, int n_text, i
 int launch_qk_prep(const void *q_in, const void *k_in, void *q_out, void *k_out, const float *gain_q, const float *gain_k,
                    int n_bh, int grid_h, int grid_w, int n_text, int head_dim, int dtype, const int axes_dim[3],
                    double theta, double ntk_factor, float eps, float q_factor, cudaStream_t stream);
+// Backward pass on the tensor cores (bf16): a query-role and a key-role launch over the plan's tile schedule, which
+// must have been built without text splits.
+int launch_bwd_tc(const clear_plan &p, const void *q, const void *k, const void *v, const void *d_out, void *dq, void *dk,
+                  void *dv, float scale, cudaStream_t stream);
 // Merge of the split-KV partial results of the text-query rows (both tensor-core kernels).
 int launch_text_combine(const clear_plan &p, void *out, cudaStream_t stream);
 

@@ -153,7 +153,7 @@ void build_tile_schedule(const Shape &s, Schedule &sch)
     const int n_lin = (int)((N + kTileTokens - 1) / kTileTokens);
     sch.n_text_tiles = (T + kTileTokens - 1) / kTileTokens;
     int chunk = n_lin, n_splits = 1;
-    if (sch.n_text_tiles > 0) {
+    if (sch.n_text_tiles > 0 && !s.no_text_split) {
         n_splits = (n_lin + kSplitTargetTiles - 1) / kSplitTargetTiles;
         chunk = (n_lin + n_splits - 1) / n_splits;
         n_splits = (n_lin + chunk - 1) / chunk;

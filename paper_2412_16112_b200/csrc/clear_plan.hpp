@@ -26,12 +26,13 @@ struct Shape {
     int part = 0;
     int q_row_begin = 0, q_row_end = 0;  // rows of the band inside the grid (band parts only)
     int text_keys = 1;                   // CLEAR_PART_BAND_TEXT: are the text tokens among the keys
+    int no_text_split = 0;               // tile schedule: one item per text tile over all its keys (backward pass)
     bool operator==(const Shape &o) const
     {
         return B == o.B && H == o.H && grid_h == o.grid_h && grid_w == o.grid_w && n_text == o.n_text &&
                head_dim == o.head_dim && radius == o.radius && dtype == o.dtype && kernel == o.kernel &&
                mask_kind == o.mask_kind && mask_param == o.mask_param && part == o.part && q_row_begin == o.q_row_begin &&
-               q_row_end == o.q_row_end && text_keys == o.text_keys;
+               q_row_end == o.q_row_end && text_keys == o.text_keys && no_text_split == o.no_text_split;
     }
 };
 
