@@ -12,9 +12,10 @@
 //               dQ += dS K (dS the tensor-memory operand, K read MN-major from the same shared-memory tile).
 //   key role    stationary K_j, V_j; streamed Q_i, dO_i with the statistics of the queries i.  S^T = K Q^T,
 //               dP^T = V dO^T; P^T and dS^T as bf16 over them; dV += P^T dO, dK += dS^T Q.
-// 128 threads own one row of the stationary tile each; one more warp issues every TMA load and every MMA.  One tile
-// of each streamed tensor is staged at a time (no overlap of loads, MMAs and the elementwise step inside a CTA): the
-// first tensor-core version of the backward pass, an order of magnitude above the CUDA-core one, not yet a tuned one.
+// 128 threads own one row of the stationary tile each; one more warp issues every TMA load and every MMA.  The
+// streamed tiles go through two stages, so the next pair travels while this one computes; the MMAs and the
+// elementwise step of a CTA still take turns: a first tensor-core version of the backward pass, far above the
+// CUDA-core one, not yet a tuned one.
 // Every wait is bounded: on expiry the CTA raises the plan's status word and leaves.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -46,7 +47,7 @@ struct BwdParams {
 };
 
 struct BwdCtrl {
-    uint64_t a_full, b_full, t_full, p_ready, o_done;
+    uint64_t a_full, b_full[2], t_full, p_ready, o_done;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -71,19 +72,6 @@ __device__ __forceinline__ void bwd_drain(uint32_t bar, uint32_t parity)
     }
 }
 
-// Token of column j of a streamed tile (clamped into the sequence: columns that do not exist are masked anyway).
-__device__ __forceinline__ long long column_token(const clear_kv_tile_t &t, int j, const BwdParams &prm)
-{
-    long long tok;
-    if (t.flags & CLEAR_TILE_LINEAR) {
-        tok = (long long)t.x + j;
-    } else {
-        const int y = min(max(t.y + (j >> 4), 0), prm.grid_h - 1), x = min(max(t.x + (j & 15), 0), prm.grid_w - 1);
-        tok = (long long)prm.n_text + (long long)y * prm.grid_w + x;
-    }
-    return min(tok, prm.n_tokens - 1);
-}
-
 template <int D, bool KEY_ROLE>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_constant__ CUtensorMap tm_a1_txt,
@@ -102,11 +90,12 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    const uint32_t sA1 = smem_base, sA2 = sA1 + kTileBytes, sB1 = sA2 + kTileBytes, sB2 = sB1 + kTileBytes;
-    BwdCtrl *ctrl = reinterpret_cast<BwdCtrl *>(smem_gen + 4 * kTileBytes);
+    // two stationary tiles, then two stages of the two streamed tiles
+    const uint32_t sA1 = smem_base, sA2 = sA1 + kTileBytes, sB = sA2 + kTileBytes;
+    BwdCtrl *ctrl = reinterpret_cast<BwdCtrl *>(smem_gen + 6 * kTileBytes);
     volatile int *abort_flag = &ctrl->abort_flag;
-    const uint32_t b_a = ptx::smem_u32(&ctrl->a_full), b_b = ptx::smem_u32(&ctrl->b_full),
-                   b_t = ptx::smem_u32(&ctrl->t_full), b_p = ptx::smem_u32(&ctrl->p_ready),
+    const uint32_t b_a = ptx::smem_u32(&ctrl->a_full), b_b0 = ptx::smem_u32(&ctrl->b_full[0]),
+                   b_b1 = ptx::smem_u32(&ctrl->b_full[1]), b_t = ptx::smem_u32(&ctrl->t_full), b_p = ptx::smem_u32(&ctrl->p_ready),
                    b_o = ptx::smem_u32(&ctrl->o_done);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -125,7 +114,8 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
     if (tid == 0) {
         ctrl->abort_flag = 0;
         ptx::mbar_init(b_a, 1);
-        ptx::mbar_init(b_b, 1);
+        ptx::mbar_init(b_b0, 1);
+        ptx::mbar_init(b_b1, 1);
         ptx::mbar_init(b_t, 1);
         ptx::mbar_init(b_p, kRowThreads);
         ptx::mbar_init(b_o, 1);
@@ -156,79 +146,80 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                         ptx::tma_load_4d(dst + h * kHalfBytes, tm_img, bar, h * 64, x, y, bh);
                 }
             };
-            auto load_streamed = [&](const clear_kv_tile_t &t) {
-                ptx::mbar_expect_tx(b_b, 2 * kTileBytes);
+            // streamed tiles go through two stages: the tiles of iteration it + 1 travel while iteration it computes
+            const int n_iters = kSweeps * n_tiles;
+            auto load_streamed = [&](int it) {
+                const clear_kv_tile_t t = tiles[it % n_tiles];
+                const uint32_t bar = (it & 1) ? b_b1 : b_b0, dst = sB + (uint32_t)(it & 1) * 2 * kTileBytes;
+                ptx::mbar_expect_tx(bar, 2 * kTileBytes);
                 const bool lin = (t.flags & CLEAR_TILE_LINEAR) != 0;
-                load_tile(sB1, b_b, &tm_b1_img, &tm_b1_lin, lin, t.x, t.y);
-                load_tile(sB2, b_b, &tm_b2_img, &tm_b2_lin, lin, t.x, t.y);
+                load_tile(dst, bar, &tm_b1_img, &tm_b1_lin, lin, t.x, t.y);
+                load_tile(dst + kTileBytes, bar, &tm_b2_img, &tm_b2_lin, lin, t.x, t.y);
                 ++b_issued;
             };
             ptx::mbar_expect_tx(b_a, 2 * kTileBytes);
             load_tile(sA1, b_a, &tm_a1_img, &tm_a1_txt, is_text, item.qx, item.qy);
             load_tile(sA2, b_a, &tm_a2_img, &tm_a2_txt, is_text, item.qx, item.qy);
-            load_streamed(tiles[0]);
+            load_streamed(0);
             a_seen = bwd_wait(b_a, 0, abort_flag, prm.status, 1);
 
-            int iter = 0, n_grad = 0;
+            int n_grad = 0;
             bool ok = a_seen;
-            for (int sweep = 0; sweep < kSweeps && ok; ++sweep) {
-                const bool grad = KEY_ROLE || sweep == 1;
-                for (int i = 0; i < n_tiles && ok; ++i, ++iter) {
-                    const uint32_t ph = (uint32_t)(iter & 1);
-                    if (!(ok = bwd_wait(b_b, ph, abort_flag, prm.status, 2))) break;
-                    ++b_seen;
+            for (int it = 0; it < n_iters && ok; ++it) {
+                const bool grad = KEY_ROLE || it >= n_tiles;
+                const uint32_t ph = (uint32_t)(it & 1);
+                const uint32_t sB1 = sB + ph * 2 * kTileBytes, sB2 = sB1 + kTileBytes;
+                // the other stage was last read by the MMAs of iteration it - 1, which have retired
+                if (it + 1 < n_iters) load_streamed(it + 1);
+                if (!(ok = bwd_wait(ph ? b_b1 : b_b0, (uint32_t)((it >> 1) & 1), abort_flag, prm.status, 2))) break;
+                ++b_seen;
+                ptx::tc_fence_after();
+                // ---- T1 = A1 B1^T, T2 = A2 B2^T : D/16 MMAs of 16 channels each ----------------------------
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                    ptx::mma_ss(tmem_T1, ptx::smem_desc_sw128(sA1 + off, 16, 1024), ptx::smem_desc_sw128(sB1 + off, 16, 1024),
+                                kIdescT, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                    ptx::mma_ss(tmem_T2, ptx::smem_desc_sw128(sA2 + off, 16, 1024), ptx::smem_desc_sw128(sB2 + off, 16, 1024),
+                                kIdescT, kk > 0);
+                }
+                ptx::tc_commit(b_t);
+                mma_pending = true;
+                // the rows have read T1, T2 (and, in a gradient sweep, put P / dS over them)
+                if (!(ok = bwd_wait(b_p, ph, abort_flag, prm.status, 3))) break;
+                mma_pending = false;
+                if (grad) {
                     ptx::tc_fence_after();
-                    // ---- T1 = A1 B1^T, T2 = A2 B2^T : D/16 MMAs of 16 channels each ------------------------
+                    // ---- the accumulators: 8 MMAs over 16 streamed tokens each, B read MN-major -------------
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                        ptx::mma_ss(tmem_T1, ptx::smem_desc_sw128(sA1 + off, 16, 1024), ptx::smem_desc_sw128(sB1 + off, 16, 1024),
-                                    kIdescT, kk > 0);
-                    }
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                        ptx::mma_ss(tmem_T2, ptx::smem_desc_sw128(sA2 + off, 16, 1024), ptx::smem_desc_sw128(sB2 + off, 16, 1024),
-                                    kIdescT, kk > 0);
-                    }
-                    ptx::tc_commit(b_t);
-                    mma_pending = true;
-                    // the rows have read T1, T2 (and, in a gradient sweep, put P / dS over them)
-                    if (!(ok = bwd_wait(b_p, ph, abort_flag, prm.status, 3))) break;
-                    mma_pending = false;
-                    if (grad) {
-                        ptx::tc_fence_after();
-                        // ---- the accumulators: 8 MMAs over 16 streamed tokens each, B read MN-major ---------
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t acc = (n_grad > 0 || kk > 0) ? 1u : 0u;
-                            if (KEY_ROLE) {
-                                ptx::mma_ts(tmem_A1, tmem_T1 + kk * 8, ptx::smem_desc_sw128(sB2 + kk * 2048, kHalfBytes, 1024),
-                                            kIdescAcc, acc);   // dV += P^T dO
-                                ptx::mma_ts(tmem_A2, tmem_T2 + kk * 8, ptx::smem_desc_sw128(sB1 + kk * 2048, kHalfBytes, 1024),
-                                            kIdescAcc, acc);   // dK += dS^T Q
-                            } else {
-                                ptx::mma_ts(tmem_A1, tmem_T1 + kk * 8, ptx::smem_desc_sw128(sB1 + kk * 2048, kHalfBytes, 1024),
-                                            kIdescAcc, acc);   // dQ += dS K
-                            }
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t acc = (n_grad > 0 || kk > 0) ? 1u : 0u;
+                        if (KEY_ROLE) {
+                            ptx::mma_ts(tmem_A1, tmem_T1 + kk * 8, ptx::smem_desc_sw128(sB2 + kk * 2048, kHalfBytes, 1024),
+                                        kIdescAcc, acc);   // dV += P^T dO
+                            ptx::mma_ts(tmem_A2, tmem_T2 + kk * 8, ptx::smem_desc_sw128(sB1 + kk * 2048, kHalfBytes, 1024),
+                                        kIdescAcc, acc);   // dK += dS^T Q
+                        } else {
+                            ptx::mma_ts(tmem_A1, tmem_T1 + kk * 8, ptx::smem_desc_sw128(sB1 + kk * 2048, kHalfBytes, 1024),
+                                        kIdescAcc, acc);   // dQ += dS K
                         }
-                        ptx::tc_commit(b_o);
-                        mma_pending = true;
-                        if (!(ok = bwd_wait(b_o, (uint32_t)(n_grad & 1), abort_flag, prm.status, 4))) break;
-                        mma_pending = false;
-                        ++n_grad;
                     }
-                    // the streamed buffers are free: next tile of this sweep, or the first one of the next sweep
-                    if (i + 1 < n_tiles)
-                        load_streamed(tiles[i + 1]);
-                    else if (sweep + 1 < kSweeps)
-                        load_streamed(tiles[0]);
+                    ptx::tc_commit(b_o);
+                    mma_pending = true;
+                    if (!(ok = bwd_wait(b_o, (uint32_t)(n_grad & 1), abort_flag, prm.status, 4))) break;
+                    mma_pending = false;
+                    ++n_grad;
                 }
             }
             if (*abort_flag) {
                 // leave nothing in flight: copies that were issued must land, MMAs must retire
                 if (!a_seen) bwd_drain(b_a, 0);
-                if (b_issued > b_seen) bwd_drain(b_b, (uint32_t)(b_seen & 1));
+                // at most two loads are in flight: iterations b_seen and b_seen + 1
+                for (int it = b_seen; it < b_issued; ++it) bwd_drain((it & 1) ? b_b1 : b_b0, (uint32_t)((it >> 1) & 1));
                 if (mma_pending) __nanosleep(100000);
             }
         }
@@ -331,6 +322,17 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                 }
 
                 // ---- gradient sweep: P = exp2(c T1 - m) / l, dS = P (T2 - delta), bf16 over T1 / T2 -------------
+                // key role: where the statistics of the tile's columns lie (a column that does not exist is masked;
+                // its address stays inside the buffer, which is padded by one tile)
+                const bool linear = (t.flags & CLEAR_TILE_LINEAR) != 0;
+                const float4 *col_stats[KEY_ROLE ? 8 : 1];
+                if (KEY_ROLE) {
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const int y = min(t.y + rr, prm.grid_h - 1);
+                        col_stats[rr] = linear ? stats + t.x : stats + prm.n_text + (long long)y * prm.grid_w + t.x;
+                    }
+                }
 #pragma unroll
                 for (int w = 0; w < 4; ++w) {
                     uint32_t s[32], g[32], pk[16], dk[16];
@@ -344,7 +346,8 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                         for (int u = 0; u < 2; ++u) {
                             float m_c, il_c, d_c;
                             if (KEY_ROLE) {
-                                const float4 st = __ldg(stats + column_token(t, 32 * w + j + u, prm));
+                                const int jj = 32 * w + j + u;
+                                const float4 st = __ldg(col_stats[linear ? 0 : (jj >> 4)] + (linear ? jj : (jj & 15)));
                                 m_c = st.x;
                                 il_c = st.y;
                                 d_c = st.z;
@@ -435,7 +438,9 @@ int launch_bwd_tc(const clear_plan &p, const void *q, const void *k, const void 
     const uint64_t d = (uint64_t)s.head_dim, gw = (uint64_t)s.grid_w, gh = (uint64_t)s.grid_h, T = (uint64_t)s.n_text;
     const uint64_t N = T + gw * gh, BH = (uint64_t)s.B * s.H;
     if (!p.d_bwd_stats) {
-        cudaError_t e = cudaMalloc((void **)&p.d_bwd_stats, (size_t)BH * N * sizeof(float4));
+        // one tile of padding: the statistics of columns past the end are read (and masked), never used
+        cudaError_t e = cudaMalloc((void **)&p.d_bwd_stats, ((size_t)BH * N + kTileTokens) * sizeof(float4));
+        if (e == cudaSuccess) e = cudaMemsetAsync(p.d_bwd_stats, 0, ((size_t)BH * N + kTileTokens) * sizeof(float4), stream);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return e == cudaErrorMemoryAllocation ? CLEAR_ERR_NO_MEMORY : CLEAR_ERR_CUDA;
@@ -492,8 +497,8 @@ int launch_bwd_tc(const clear_plan &p, const void *q, const void *k, const void 
         return CLEAR_OK;
     };
     if (s.head_dim == 128)
-        return run(clear_bwd_tc_kernel<128, false>, clear_bwd_tc_kernel<128, true>, 4 * 32768 + 1024 + sizeof(BwdCtrl));
-    return run(clear_bwd_tc_kernel<64, false>, clear_bwd_tc_kernel<64, true>, 4 * 16384 + 1024 + sizeof(BwdCtrl));
+        return run(clear_bwd_tc_kernel<128, false>, clear_bwd_tc_kernel<128, true>, 6 * 32768 + 1024 + sizeof(BwdCtrl));
+    return run(clear_bwd_tc_kernel<64, false>, clear_bwd_tc_kernel<64, true>, 6 * 16384 + 1024 + sizeof(BwdCtrl));
 }
 
 }  // namespace clear
