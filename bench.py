@@ -8,7 +8,7 @@ Prints ONE JSON line.  `value` is effective TFLOP/s, 4 * sum(M) * head_dim * H *
 entry point with the host<->device copies inside the timed region.  With N > 1 (torchrun) every rank runs
 an independent replica of the workload on its own GPU: the path has no exchange step.
 `qk_prep` times, outside `value`, the one-pass Q/K preparation kernel (normalisation + rotary embedding) on the
-same shape against the HBM copy rate.
+same shape against the HBM copy rate; `bwd` times the tensor-core backward pass of the operator.
 `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload (rank 0 only).
 """
 from __future__ import annotations
@@ -392,6 +392,29 @@ def run_ours(args, w):
                    "note": "tensors fit in L2: no HBM figure" if small else "tensors larger than L2"}
         del k_out
 
+    # ---- the backward pass of the same operator on the tensor cores (outside `value`) ---------------------
+    bwd = None
+    if not args.no_bwd and w.dtype == "bf16" and w.head_dim in (64, 128):
+        grads = [torch.empty_like(qd) for _ in range(3)]
+        n_bwd = 3
+        for _ in range(2):
+            clear.clear_attn_bwd_bf16_tc(qd, kd, vd, vd, *grads, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale)
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        b0.record(stream)
+        for _ in range(n_bwd):
+            clear.clear_attn_bwd_bf16_tc(qd, kd, vd, vd, *grads, w.grid_h, w.grid_w, w.n_text, w.radius, w.scale)
+        b1.record(stream)
+        torch.cuda.synchronize()
+        clear.clear_cache_check()
+        bwd_ms = b0.elapsed_time(b1) / n_bwd
+        bwd_flops = 2.5 * flops   # five matrix products per allowed pair against the forward's two
+        bwd = {"kernel": "clear_bwd_tc_kernel (query role + key role)", "ms": bwd_ms, "flops_per_call": bwd_flops,
+               "value": bwd_flops / (bwd_ms * 1e-3) / 1e12, "unit": "effective TFLOP/s (10*sum(M)*c)",
+               "frac": bwd_flops / (bwd_ms * 1e-3) / 1e12 / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
+               "launches": 2 * n_bwd, "note": "upstream gradient = v (any bf16 data of the right shape)"}
+        del grads
+
     cpu_baseline = None
     if not args.no_cpu:
         if w.name in FULL_ORACLE_WORKLOADS:
@@ -410,7 +433,7 @@ def run_ours(args, w):
             "ms_min": float(min(ms)), "ms_median": float(np.median(ms)), "wall_s_timed_region": t_wall,
             "ms_x_sm_mhz": ms_per_step * clock_info["sm_mhz"] if clock_info.get("sm_mhz") else None,
             "flops_per_call": flops, "sum_mask_per_head": info.sum_mask, "parallelism": "replicas",
-            "qk_prep": qk_prep}
+            "qk_prep": qk_prep, "bwd": bwd}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -514,6 +537,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-prep", action="store_true", help="skip the timing of the Q/K preparation kernel")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-bwd", action="store_true", help="skip the timing of the tensor-core backward pass")
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "bands"],
                     help="replicas (default): every rank runs the whole workload; bands: one workload cut into row "
                          "bands over the ranks (Sec. 3.4), strong scaling")
