@@ -12,7 +12,8 @@
 //               dQ += dS K (dS the tensor-memory operand, K read MN-major from the same shared-memory tile).
 //   key role    stationary K_j, V_j; streamed Q_i, dO_i with the statistics of the queries i.  S^T = K Q^T,
 //               dP^T = V dO^T; P^T and dS^T as bf16 over them; dV += P^T dO, dK += dS^T Q.
-// 128 threads own one row of the stationary tile each; one more warp issues every TMA load and every MMA.  The
+// 256 threads: two per row of the stationary tile, each with half of the columns of a streamed tile (the halves of
+// a row merge their softmax statistics once, after sweep 1); one more warp issues every TMA load and every MMA.  The
 // streamed tiles go through two stages, so the next pair travels while this one computes; the MMAs and the
 // elementwise step of a CTA still take turns: a first tensor-core version of the backward pass, far above the
 // CUDA-core one, not yet a tuned one.
@@ -28,8 +29,9 @@
 namespace clear {
 namespace {
 
-constexpr int kRowThreads = 128;
-constexpr int kBwdThreads = 160;         // 4 row warps + 1 control warp (TMA + MMA issue)
+constexpr int kRowThreads = 256;         // two threads per row of the stationary tile: one per half of the columns
+constexpr int kControlWarp = 8;
+constexpr int kBwdThreads = 288;         // 8 row warps + 1 control warp (TMA + MMA issue)
 constexpr uint32_t kBwdTmemCols = 512;   // T1 | T2 | ACC1 | ACC2, 128 columns each
 constexpr uint32_t kBwdSpinLimit = 1u << 22;
 
@@ -47,7 +49,8 @@ struct BwdParams {
 };
 
 struct BwdCtrl {
-    uint64_t a_full, b_full[2], t_full, p_ready, o_done;
+    uint64_t a_full, b_full[2], t_full, p_ready, o_done, x_done;
+    float4 part[2][128];   // query role: the two halves' row statistics after sweep 1
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -96,7 +99,7 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
     volatile int *abort_flag = &ctrl->abort_flag;
     const uint32_t b_a = ptx::smem_u32(&ctrl->a_full), b_b0 = ptx::smem_u32(&ctrl->b_full[0]),
                    b_b1 = ptx::smem_u32(&ctrl->b_full[1]), b_t = ptx::smem_u32(&ctrl->t_full), b_p = ptx::smem_u32(&ctrl->p_ready),
-                   b_o = ptx::smem_u32(&ctrl->o_done);
+                   b_o = ptx::smem_u32(&ctrl->o_done), b_x = ptx::smem_u32(&ctrl->x_done);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.y;
@@ -119,9 +122,10 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
         ptx::mbar_init(b_t, 1);
         ptx::mbar_init(b_p, kRowThreads);
         ptx::mbar_init(b_o, 1);
+        ptx::mbar_init(b_x, kRowThreads);
         ptx::fence_mbar_init();
     }
-    if (warp == 4) {
+    if (warp == kControlWarp) {
         ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), kBwdTmemCols);
         ptx::tmem_relinquish();
     }
@@ -131,7 +135,7 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
     const uint32_t tmem = ctrl->tmem_base;
     const uint32_t tmem_T1 = tmem, tmem_T2 = tmem + 128, tmem_A1 = tmem + 256, tmem_A2 = tmem + 384;
 
-    if (warp == 4) {
+    if (warp == kControlWarp) {
         // ================= control warp: one lane issues every TMA load and every MMA ====================
         if (lane == 0) {
             int b_issued = 0, b_seen = 0;
@@ -199,12 +203,12 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t acc = (n_grad > 0 || kk > 0) ? 1u : 0u;
                         if (KEY_ROLE) {
-                            ptx::mma_ts(tmem_A1, tmem_T1 + kk * 8, ptx::smem_desc_sw128(sB2 + kk * 2048, kHalfBytes, 1024),
+                            ptx::mma_ts(tmem_A1, tmem_T1 + (kk >> 2) * 64 + (kk & 3) * 8, ptx::smem_desc_sw128(sB2 + kk * 2048, kHalfBytes, 1024),
                                         kIdescAcc, acc);   // dV += P^T dO
-                            ptx::mma_ts(tmem_A2, tmem_T2 + kk * 8, ptx::smem_desc_sw128(sB1 + kk * 2048, kHalfBytes, 1024),
+                            ptx::mma_ts(tmem_A2, tmem_T2 + (kk >> 2) * 64 + (kk & 3) * 8, ptx::smem_desc_sw128(sB1 + kk * 2048, kHalfBytes, 1024),
                                         kIdescAcc, acc);   // dK += dS^T Q
                         } else {
-                            ptx::mma_ts(tmem_A1, tmem_T1 + kk * 8, ptx::smem_desc_sw128(sB1 + kk * 2048, kHalfBytes, 1024),
+                            ptx::mma_ts(tmem_A1, tmem_T1 + (kk >> 2) * 64 + (kk & 3) * 8, ptx::smem_desc_sw128(sB1 + kk * 2048, kHalfBytes, 1024),
                                         kIdescAcc, acc);   // dQ += dS K
                         }
                     }
@@ -225,9 +229,12 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
         }
         __syncwarp();
     } else {
-        // ================= row warps: thread r owns row r of the stationary tile ============================
-        const int r = tid;
-        const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+        // ================= row warps: thread (g, r) owns row r of the stationary tile and the columns
+        // [64 g, 64 g + 64) of every streamed tile (two warps per tensor-memory lane quadrant) =================
+        const int g = warp >> 2;                 // column half
+        const int r = (warp & 3) * 32 + lane;    // row of the tile
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t col0 = 64u * (uint32_t)g;  // first fp32 column of this thread's half; its bf16 results go there too
         const float c = prm.scale_log2;
         int q_y = 0, q_x = 0;
         bool row_valid;
@@ -242,7 +249,8 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
             row_token = (long long)prm.n_text + (long long)q_y * prm.grid_w + q_x;
         }
         float4 *stats = prm.stats + (long long)bh * prm.n_tokens;
-        // query role: the row's own statistics; running values in sweep 1 (m in log2 units, scale included)
+        // query role: statistics of the row; in sweep 1 running values over THIS thread's columns only (m in log2
+        // units, scale included), merged with the other half's at the end of the sweep
         float m_row = -INFINITY, l_row = 0.f, d_row = 0.f, il_row = 0.f;
         bool alive = true;
         int iter = 0, n_grad = 0;
@@ -252,22 +260,21 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
             for (int i = 0; i < n_tiles; ++i, ++iter) {
                 const uint32_t ph = (uint32_t)(iter & 1);
                 const clear_kv_tile_t t = tiles[i];
-                // ---- mask bits of this row for the tile (bit j = column j allowed; the mask is symmetric, so the
-                // row's token plays the query whichever role the kernel runs in) --------------------------------
-                uint32_t mw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+                // ---- mask bits of this row for its 64 columns (bit j of word w = column 64 g + 32 w + j allowed; the
+                // mask is symmetric, so the row's token plays the query whichever role the kernel runs in) ----------
+                uint32_t mw[2] = {0xffffffffu, 0xffffffffu};
                 if (t.flags & CLEAR_TILE_MASKED) {
                     if (t.flags & CLEAR_TILE_LINEAR) {
 #pragma unroll
-                        for (int w = 0; w < 4; ++w) {
-                            const int n = min(max(t.n_valid - 32 * w, 0), 32);
+                        for (int w = 0; w < 2; ++w) {
+                            const int n = min(max(t.n_valid - 64 * g - 32 * w, 0), 32);
                             mw[w] = n == 32 ? 0xffffffffu : ((1u << n) - 1u);
                         }
                     } else {
+                        mw[0] = mw[1] = 0u;
 #pragma unroll
-                        for (int w = 0; w < 4; ++w) mw[w] = 0u;
-#pragma unroll
-                        for (int rr = 0; rr < 8; ++rr) {
-                            const int ky = t.y + rr;
+                        for (int rr = 0; rr < 4; ++rr) {
+                            const int ky = t.y + 4 * g + rr;
                             const int ady = abs(ky - q_y);
                             uint32_t bits = 0u;
                             if (row_valid && ky >= 0 && ky < prm.grid_h && ady < prm.n_half_width) {
@@ -286,12 +293,12 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                 ptx::tc_fence_after();
 
                 if (!grad) {
-                    // ---- sweep 1 of the query role: online softmax statistics and delta ------------------------
+                    // ---- sweep 1 of the query role: online softmax statistics and delta over this half ----------
                     float mx = -INFINITY;
 #pragma unroll
-                    for (int w = 0; w < 4; ++w) {
+                    for (int w = 0; w < 2; ++w) {
                         uint32_t s[32];
-                        ptx::tmem_ld32(tmem_T1 + lane_off + 32 * w, s);
+                        ptx::tmem_ld32(tmem_T1 + lane_off + col0 + 32 * w, s);
                         ptx::tmem_wait_ld();
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
@@ -303,16 +310,16 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                     d_row *= alpha;
                     const float mc = (m_new == -INFINITY) ? 0.f : m_new;
 #pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        uint32_t s[32], g[32];
-                        ptx::tmem_ld32(tmem_T1 + lane_off + 32 * w, s);
-                        ptx::tmem_ld32(tmem_T2 + lane_off + 32 * w, g);
+                    for (int w = 0; w < 2; ++w) {
+                        uint32_t s[32], gg[32];
+                        ptx::tmem_ld32(tmem_T1 + lane_off + col0 + 32 * w, s);
+                        ptx::tmem_ld32(tmem_T2 + lane_off + col0 + 32 * w, gg);
                         ptx::tmem_wait_ld();
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             const float p = ((mw[w] >> j) & 1u) ? ptx::ex2(fmaf(__uint_as_float(s[j]), c, -mc)) : 0.f;
                             l_row += p;
-                            d_row = fmaf(p, __uint_as_float(g[j]), d_row);
+                            d_row = fmaf(p, __uint_as_float(gg[j]), d_row);
                         }
                     }
                     m_row = m_new;
@@ -325,19 +332,19 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                 // key role: where the statistics of the tile's columns lie (a column that does not exist is masked;
                 // its address stays inside the buffer, which is padded by one tile)
                 const bool linear = (t.flags & CLEAR_TILE_LINEAR) != 0;
-                const float4 *col_stats[KEY_ROLE ? 8 : 1];
+                const float4 *col_stats[KEY_ROLE ? 4 : 1];
                 if (KEY_ROLE) {
 #pragma unroll
-                    for (int rr = 0; rr < 8; ++rr) {
-                        const int y = min(t.y + rr, prm.grid_h - 1);
-                        col_stats[rr] = linear ? stats + t.x : stats + prm.n_text + (long long)y * prm.grid_w + t.x;
+                    for (int rr = 0; rr < 4; ++rr) {
+                        const int y = min(t.y + 4 * g + rr, prm.grid_h - 1);
+                        col_stats[rr] = linear ? stats + t.x + 64 * g : stats + prm.n_text + (long long)y * prm.grid_w + t.x;
                     }
                 }
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    uint32_t s[32], g[32], pk[16], dk[16];
-                    ptx::tmem_ld32(tmem_T1 + lane_off + 32 * w, s);
-                    ptx::tmem_ld32(tmem_T2 + lane_off + 32 * w, g);
+                for (int w = 0; w < 2; ++w) {
+                    uint32_t s[32], gg[32], pk[16], dk[16];
+                    ptx::tmem_ld32(tmem_T1 + lane_off + col0 + 32 * w, s);
+                    ptx::tmem_ld32(tmem_T2 + lane_off + col0 + 32 * w, gg);
                     ptx::tmem_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
@@ -346,7 +353,7 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                         for (int u = 0; u < 2; ++u) {
                             float m_c, il_c, d_c;
                             if (KEY_ROLE) {
-                                const int jj = 32 * w + j + u;
+                                const int jj = 32 * w + j + u;  // column within this thread's half
                                 const float4 st = __ldg(col_stats[linear ? 0 : (jj >> 4)] + (linear ? jj : (jj & 15)));
                                 m_c = st.x;
                                 il_c = st.y;
@@ -358,17 +365,18 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                             }
                             const bool on = ((mw[w] >> (j + u)) & 1u) != 0u;
                             p[u] = on ? ptx::ex2(fmaf(__uint_as_float(s[j + u]), c, -m_c)) * il_c : 0.f;
-                            ds[u] = p[u] * (__uint_as_float(g[j + u]) - d_c);
+                            ds[u] = p[u] * (__uint_as_float(gg[j + u]) - d_c);
                         }
                         pk[j >> 1] = ptx::pack_bf16(p[0], p[1]);
                         dk[j >> 1] = ptx::pack_bf16(ds[0], ds[1]);
                     }
-                    // columns [16 w, 16 w + 16) of a region lie inside its fp32 chunk w / 2, which is in registers
+                    // the half's 32 bf16 columns sit at the start of its own fp32 columns, all of which this thread
+                    // has in registers before it writes (chunk 0 covers them)
                     if (KEY_ROLE) {
-                        ptx::tmem_st16(tmem_T1 + lane_off + 16 * w, pk);
-                        ptx::tmem_st16(tmem_T2 + lane_off + 16 * w, dk);
+                        ptx::tmem_st16(tmem_T1 + lane_off + col0 + 16 * w, pk);
+                        ptx::tmem_st16(tmem_T2 + lane_off + col0 + 16 * w, dk);
                     } else {
-                        ptx::tmem_st16(tmem_T1 + lane_off + 16 * w, dk);
+                        ptx::tmem_st16(tmem_T1 + lane_off + col0 + 16 * w, dk);
                     }
                 }
                 ptx::tmem_wait_st();
@@ -377,15 +385,23 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                 ++n_grad;
             }
             if (!KEY_ROLE && sweep == 0 && alive) {
-                // the row's statistics: kept for sweep 2, and left for the key role
-                il_row = l_row > 0.f ? 1.f / l_row : 0.f;
-                d_row *= il_row;
-                if (m_row == -INFINITY) m_row = 0.f;  // a row without any key: P = 0 through il = 0
-                if (row_valid) stats[row_token] = make_float4(m_row, il_row, d_row, 0.f);
+                // the two halves of a row merge their statistics (a split softmax); kept for sweep 2, and left in
+                // global memory for the key role
+                ctrl->part[g][r] = make_float4(m_row, l_row, d_row, 0.f);
+                ptx::mbar_arrive(b_x);
+                if (!__all_sync(0xffffffffu, bwd_wait(b_x, 0, abort_flag, prm.status, 7))) { alive = false; break; }
+                const float4 o = ctrl->part[g ^ 1][r];
+                const float m = fmaxf(m_row, o.x);
+                const float a0 = (m_row == -INFINITY) ? 0.f : ptx::ex2(m_row - m), a1 = (o.x == -INFINITY) ? 0.f : ptx::ex2(o.x - m);
+                const float l = l_row * a0 + o.y * a1;
+                il_row = l > 0.f ? 1.f / l : 0.f;
+                d_row = (d_row * a0 + o.z * a1) * il_row;
+                m_row = (m == -INFINITY) ? 0.f : m;  // a row without any key: P = 0 through il = 0
+                if (row_valid && g == 0) stats[row_token] = make_float4(m_row, il_row, d_row, 0.f);
             }
         }
 
-        // ---- epilogue: wait for the last accumulation, then store the rows --------------------------------------
+        // ---- epilogue: wait for the last accumulation, then store the rows (each half its share of the channels) ----
         if (alive && n_grad > 0)
             alive = __all_sync(0xffffffffu, bwd_wait(b_o, (uint32_t)((n_grad - 1) & 1), abort_flag, prm.status, 6));
         if (alive) {
@@ -393,7 +409,8 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
             auto store_rows = [&](uint32_t tmem_acc, __nv_bfloat16 *dst_base, float factor) {
                 __nv_bfloat16 *dst = dst_base + ((long long)bh * prm.n_tokens + row_token) * D;
 #pragma unroll
-                for (int w = 0; w < D / 32; ++w) {
+                for (int ww = 0; ww < D / 64; ++ww) {
+                    const int w = g * (D / 64) + ww;  // 32-channel chunk
                     uint32_t o[32];
                     ptx::tmem_ld32(tmem_acc + lane_off + 32 * w, o);
                     ptx::tmem_wait_ld();
@@ -421,7 +438,7 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
 
     ptx::tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kControlWarp) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem, kBwdTmemCols);
     }
