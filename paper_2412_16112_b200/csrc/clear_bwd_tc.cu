@@ -165,20 +165,16 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
             load_tile(sA1, b_a, &tm_a1_img, &tm_a1_txt, is_text, item.qx, item.qy);
             load_tile(sA2, b_a, &tm_a2_img, &tm_a2_txt, is_text, item.qx, item.qy);
             load_streamed(0);
+            if (n_iters > 1) load_streamed(1);
             a_seen = bwd_wait(b_a, 0, abort_flag, prm.status, 1);
 
-            int n_grad = 0;
-            bool ok = a_seen;
-            for (int it = 0; it < n_iters && ok; ++it) {
-                const bool grad = KEY_ROLE || it >= n_tiles;
+            // T1 = A1 B1^T, T2 = A2 B2^T of iteration it: D/16 MMAs of 16 channels each
+            auto issue_t = [&](int it) -> bool {
                 const uint32_t ph = (uint32_t)(it & 1);
                 const uint32_t sB1 = sB + ph * 2 * kTileBytes, sB2 = sB1 + kTileBytes;
-                // the other stage was last read by the MMAs of iteration it - 1, which have retired
-                if (it + 1 < n_iters) load_streamed(it + 1);
-                if (!(ok = bwd_wait(ph ? b_b1 : b_b0, (uint32_t)((it >> 1) & 1), abort_flag, prm.status, 2))) break;
+                if (!bwd_wait(ph ? b_b1 : b_b0, (uint32_t)((it >> 1) & 1), abort_flag, prm.status, 2)) return false;
                 ++b_seen;
                 ptx::tc_fence_after();
-                // ---- T1 = A1 B1^T, T2 = A2 B2^T : D/16 MMAs of 16 channels each ----------------------------
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
@@ -193,6 +189,15 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                 }
                 ptx::tc_commit(b_t);
                 mma_pending = true;
+                return true;
+            };
+
+            int n_grad = 0;
+            bool ok = a_seen && issue_t(0);
+            for (int it = 0; it < n_iters && ok; ++it) {
+                const bool grad = KEY_ROLE || it >= n_tiles;
+                const uint32_t ph = (uint32_t)(it & 1);
+                const uint32_t sB1 = sB + ph * 2 * kTileBytes, sB2 = sB1 + kTileBytes;
                 // the rows have read T1, T2 (and, in a gradient sweep, put P / dS over them)
                 if (!(ok = bwd_wait(b_p, ph, abort_flag, prm.status, 3))) break;
                 mma_pending = false;
@@ -214,10 +219,17 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                     }
                     ptx::tc_commit(b_o);
                     mma_pending = true;
+                }
+                // the next tile's T1, T2 go behind these MMAs on the same pipe: they overwrite P / dS only after the
+                // accumulations have read them, and run while this warp waits below
+                if (it + 1 < n_iters && !(ok = issue_t(it + 1))) break;
+                if (grad) {
                     if (!(ok = bwd_wait(b_o, (uint32_t)(n_grad & 1), abort_flag, prm.status, 4))) break;
-                    mma_pending = false;
+                    if (it + 1 >= n_iters) mma_pending = false;
                     ++n_grad;
                 }
+                // this iteration's stage is free (its MMAs have retired): the tiles of iteration it + 2 may land in it
+                if (it + 2 < n_iters) load_streamed(it + 2);
             }
             if (*abort_flag) {
                 // leave nothing in flight: copies that were issued must land, MMAs must retire
