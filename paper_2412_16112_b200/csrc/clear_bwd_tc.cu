@@ -50,7 +50,9 @@ struct BwdParams {
 
 struct BwdCtrl {
     uint64_t a_full, b_full[2], t_full, p_ready, o_done, x_done;
+    uint64_t s_ready;
     float4 part[2][128];   // query role: the two halves' row statistics after sweep 1
+    float4 col[2][128];    // key role: statistics of the streamed tile's 128 columns, two stages
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -99,7 +101,8 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
     volatile int *abort_flag = &ctrl->abort_flag;
     const uint32_t b_a = ptx::smem_u32(&ctrl->a_full), b_b0 = ptx::smem_u32(&ctrl->b_full[0]),
                    b_b1 = ptx::smem_u32(&ctrl->b_full[1]), b_t = ptx::smem_u32(&ctrl->t_full), b_p = ptx::smem_u32(&ctrl->p_ready),
-                   b_o = ptx::smem_u32(&ctrl->o_done), b_x = ptx::smem_u32(&ctrl->x_done);
+                   b_o = ptx::smem_u32(&ctrl->o_done), b_x = ptx::smem_u32(&ctrl->x_done),
+                   b_s = ptx::smem_u32(&ctrl->s_ready);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.y;
@@ -123,6 +126,7 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
         ptx::mbar_init(b_p, kRowThreads);
         ptx::mbar_init(b_o, 1);
         ptx::mbar_init(b_x, kRowThreads);
+        ptx::mbar_init(b_s, 128);
         ptx::fence_mbar_init();
     }
     if (warp == kControlWarp) {
@@ -300,8 +304,22 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                     }
                 }
 
+                // key role: the statistics of the tile's 128 columns go to shared memory once, fetched by the first
+                // half's threads while the MMAs run (a column that does not exist is masked; its address stays inside
+                // the buffer, which is padded by one tile)
+                if (KEY_ROLE && g == 0) {
+                    const float4 *src;
+                    if (t.flags & CLEAR_TILE_LINEAR)
+                        src = stats + t.x + r;
+                    else
+                        src = stats + prm.n_text + (long long)min(t.y + (r >> 4), prm.grid_h - 1) * prm.grid_w + t.x + (r & 15);
+                    ctrl->col[ph][r] = __ldg(src);
+                    ptx::mbar_arrive(b_s);
+                }
+
                 // warp-uniform outcome: the tcgen05.ld / st below need the whole warp
                 if (!__all_sync(0xffffffffu, bwd_wait(b_t, ph, abort_flag, prm.status, 5))) { alive = false; break; }
+                if (KEY_ROLE && !__all_sync(0xffffffffu, bwd_wait(b_s, ph, abort_flag, prm.status, 8))) { alive = false; break; }
                 ptx::tc_fence_after();
 
                 if (!grad) {
@@ -341,17 +359,6 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                 }
 
                 // ---- gradient sweep: P = exp2(c T1 - m) / l, dS = P (T2 - delta), bf16 over T1 / T2 -------------
-                // key role: where the statistics of the tile's columns lie (a column that does not exist is masked;
-                // its address stays inside the buffer, which is padded by one tile)
-                const bool linear = (t.flags & CLEAR_TILE_LINEAR) != 0;
-                const float4 *col_stats[KEY_ROLE ? 4 : 1];
-                if (KEY_ROLE) {
-#pragma unroll
-                    for (int rr = 0; rr < 4; ++rr) {
-                        const int y = min(t.y + 4 * g + rr, prm.grid_h - 1);
-                        col_stats[rr] = linear ? stats + t.x + 64 * g : stats + prm.n_text + (long long)y * prm.grid_w + t.x;
-                    }
-                }
 #pragma unroll
                 for (int w = 0; w < 2; ++w) {
                     uint32_t s[32], gg[32], pk[16], dk[16];
@@ -365,8 +372,7 @@ clear_bwd_tc_kernel(const __grid_constant__ CUtensorMap tm_a1_img, const __grid_
                         for (int u = 0; u < 2; ++u) {
                             float m_c, il_c, d_c;
                             if (KEY_ROLE) {
-                                const int jj = 32 * w + j + u;  // column within this thread's half
-                                const float4 st = __ldg(col_stats[linear ? 0 : (jj >> 4)] + (linear ? jj : (jj & 15)));
+                                const float4 st = ctrl->col[ph][64 * g + 32 * w + j + u];
                                 m_c = st.x;
                                 il_c = st.y;
                                 d_c = st.z;
